@@ -1,0 +1,161 @@
+/*
+ * rapid3.h -- C ABI of the policy-gated block-sparse joint attention library (sm_100a).
+ *
+ * The hot path is the one the Sparse-Attention policy head of RAPID^3 accelerates
+ * (paper Sec. 3.2 "Level-3: Sparse-Attention", Sec. 3.3 c): inside each MMDiT block of a
+ * denoising step the joint (text + image token) self-attention is replaced by a sparse
+ * attention whose sparsity level is chosen per image and per step by the policy; an image
+ * whose Step-Skip (Sec. 3.2 "Level-1") or Cache-Reuse (Sec. 3.2 "Level-2", Sec. 3.3 b)
+ * action fires runs no attention at all in that step.
+ *
+ * Sparsity rule (the paper leaves it to a third-party kernel; this library fixes it):
+ *   - the joint sequence is text tokens first, then image tokens in raster order;
+ *     it is cut into blocks of 64 tokens, nb = ceil(N / 64); the last block may be short;
+ *   - block scores S[i][j] = mean(Q over block i) . mean(K over block j)   (no softmax scale);
+ *   - a block that holds at least one text token is a "text block" (the first ceil(n_text/64));
+ *   - query block i always keeps: every text block, and block i itself; a text query block
+ *     keeps every block;
+ *   - of its other ("free") blocks it keeps the k = min(n_free, ceil(ratio * n_free - 1e-6))
+ *     with the highest score, ties broken towards the lower block index;
+ *   - attention of a query token = softmax over exactly the valid tokens of the kept key
+ *     blocks of its query block, times V.
+ *
+ * Conventions
+ *   - Every `q`, `k`, `v`, `out`, `scores`, `bitmask`, `kept_idx`, `kept_cnt` pointer is a DEVICE
+ *     pointer owned by the caller.  Every `*_host` pointer is a HOST pointer that is read
+ *     before the call returns.
+ *   - Q, K, V, O are bf16 tensors [B, H, N, D] addressed with the element strides of
+ *     rapid3_shape (the D stride is 1).  Base pointers and row starts must be 16-byte aligned
+ *     (strides multiples of 8 elements).
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*), never synchronise
+ *     the host, and allocate nothing: all device workspace is created by rapid3_create.
+ *     (Exception, documented below: rapid3_gated_step_host stages through buffers it creates
+ *     on first use.)
+ *   - Every function returns a status code; nothing throws, prints or aborts.  Problems that
+ *     only the device can see (a bounded wait that ran out, a kept-list entry out of range)
+ *     are recorded in a device status word, read with rapid3_last_status.
+ *   - Non-finite inputs give undefined results.
+ */
+#ifndef RAPID3_H_
+#define RAPID3_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rapid3_ctx rapid3_ctx; /* opaque: workspace, tensor-map cache, status word */
+
+typedef struct rapid3_shape {
+    int32_t B_max;    /* largest batch a call may pass (1..64)                        */
+    int32_t H;        /* heads                                                        */
+    int32_t D;        /* head dimension: 64 or 128                                    */
+    int32_t n_text;   /* text tokens (>= 0), first in the joint sequence              */
+    int32_t n_image;  /* image tokens (>= 0), after the text tokens; N = n_text+n_image, 1..65536 */
+    int32_t block;    /* must be 64                                                   */
+    int64_t stride_b; /* element strides of Q, K, V and O; all four tensors share them */
+    int64_t stride_h;
+    int64_t stride_n;
+} rapid3_shape;
+
+enum {
+    RAPID3_OK = 0,
+    RAPID3_ERR_INVALID_ARG = -1, /* null pointer, bad count, ratio outside (0, 1], ...   */
+    RAPID3_ERR_UNSUPPORTED = -2, /* shape the kernels do not cover                       */
+    RAPID3_ERR_WORKSPACE = -3,   /* device allocation failed / size limit exceeded       */
+    RAPID3_ERR_CUDA = -4,        /* a CUDA runtime or driver call failed                 */
+    RAPID3_ERR_TIMEOUT = -5,     /* device status: a bounded wait inside a kernel ran out */
+    RAPID3_ERR_BAD_LIST = -6     /* device status: a kept-list entry was out of range    */
+};
+
+/* Per-image policy action of one step (Sec. 3.3: a^cache = 1 is a reuse, a skipped time
+ * step never runs; only ATTEND launches attention work). */
+enum { RAPID3_ACT_SKIP = 0, RAPID3_ACT_REUSE = 1, RAPID3_ACT_ATTEND = 2 };
+
+/* Creates a context for one shape on the current device and allocates all device workspace
+ * (pooled means, scores, masks and kept lists for B_max images).  *out is NULL on failure. */
+int rapid3_create(rapid3_ctx** out, const rapid3_shape* shape);
+/* Frees the workspace.  The caller makes sure no call using the context is still running. */
+int rapid3_destroy(rapid3_ctx* ctx);
+const char* rapid3_strerror(int code);
+
+/* nb = ceil((n_text + n_image) / 64) and the number of uint64 words of one bitmask row. */
+int rapid3_num_blocks(const rapid3_shape* shape);
+int rapid3_mask_words(const rapid3_shape* shape);
+
+/*
+ * Stage (a), part 1: pooled block scores (sparsity rule above, steps "block scores").
+ * For the n_img images whose batch indices are listed in img_idx_host (NULL means
+ * 0..n_img-1), writes scores[p][h][i][j] (fp32, [n_img, H, nb, nb], compacted in list order).
+ * Block means and the dot products are accumulated in fp64 and rounded once to fp32.
+ * Reads Q and K once.
+ */
+int rapid3_block_scores(rapid3_ctx* ctx, const void* q, const void* k, const int32_t* img_idx_host,
+                        int n_img, float* scores, void* stream);
+
+/*
+ * Stage (a), part 2: per (image, head, query block) forced + top-k block mask at each image's
+ * keep ratio (keep_ratio_host[p] in (0, 1]).  Outputs, all compacted like `scores`:
+ *   bitmask  [n_img, H, nb, words] uint64: bit (j % 64) of word (j / 64) set <=> query block i
+ *            attends key block j; bits >= nb are zero;
+ *   kept_idx [n_img, H, nb, nb] int32: the kept key blocks of row i in ascending order,
+ *            entries past the count are -1;
+ *   kept_cnt [n_img, H, nb] int32.
+ * The comparison is done on the fp32 scores; equal scores keep the lower block index.
+ */
+int rapid3_select_mask(rapid3_ctx* ctx, const float* scores, const float* keep_ratio_host, int n_img,
+                       uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, void* stream);
+
+/*
+ * Stage (b): masked flash-style attention over the kept tiles only.  For image p of the list
+ * (batch index img_idx_host[p], or p when the list is NULL) the kept key blocks of query block
+ * i are kept_idx[p][h][i][0 .. kept_cnt[p][h][i]).  kept_idx == NULL means every block is kept
+ * (dense attention) for all listed images.  Writes out[b][h][n][:] (bf16) for every token of
+ * the listed images and touches nothing else.  bf16 tensor-core products, fp32 online softmax.
+ * softmax_scale multiplies q.k before the softmax.
+ */
+int rapid3_sparse_joint_attn(rapid3_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                             const int32_t* img_idx_host, int n_img, const int32_t* kept_idx,
+                             const int32_t* kept_cnt, float softmax_scale, void* stream);
+
+/*
+ * One policy-gated step over a batch of B <= B_max images: action_host[b] in
+ * {SKIP, REUSE, ATTEND}; only ATTEND images are processed, at keep_ratio_host[b] in (0, 1]
+ * (ignored for the others).  Images with keep ratio exactly 1 skip the scoring and selection
+ * passes.  Skipped and reusing images launch no work and their rows of `out` stay untouched.
+ * Scores, masks and kept lists of the sparse images live in the context's workspace
+ * (see rapid3_workspace), compacted in ascending batch order of the sparse images.
+ */
+int rapid3_gated_step(rapid3_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                      const int32_t* action_host, const float* keep_ratio_host, int B,
+                      float softmax_scale, void* stream);
+
+/*
+ * The same step with HOST tensors (pinned memory recommended): copies Q, K, V of the attending
+ * images to device staging buffers, runs rapid3_gated_step and copies their rows of `out` back,
+ * all on `stream`; gated images move no bytes.  The staging buffers (4 tensors of
+ * B_max*H*N*D bf16, contiguous [B, H, N, D]; the host tensors must be contiguous too) are
+ * allocated on the first call of a context, so make that call outside any timed region.
+ * bytes_h2d / bytes_d2h (may be NULL) receive the bytes moved.
+ */
+int rapid3_gated_step_host(rapid3_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
+                           void* out_host, const int32_t* action_host, const float* keep_ratio_host, int B,
+                           float softmax_scale, void* stream, int64_t* bytes_h2d, int64_t* bytes_d2h);
+
+/* Device pointers of the workspace rapid3_gated_step fills (any may be NULL): layouts as in
+ * rapid3_block_scores / rapid3_select_mask with n_img = number of sparse images of the last step. */
+int rapid3_workspace(rapid3_ctx* ctx, float** scores, uint64_t** bitmask, int32_t** kept_idx,
+                     int32_t** kept_cnt);
+
+/* Number of kernels this context has launched so far (all entry points). */
+int64_t rapid3_launch_count(rapid3_ctx* ctx);
+
+/* Copies the device status word to *device_status (RAPID3_OK or a negative code) and clears it.
+ * Synchronises the device; call it after the stream has been synchronised. */
+int rapid3_last_status(rapid3_ctx* ctx, int* device_status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAPID3_H_ */

@@ -1,0 +1,215 @@
+"""ctypes binding of librapid3.so: argument marshalling only.
+
+Every step of the path runs in the CUDA kernels behind the C ABI (include/rapid3.h); torch is
+used for device memory and streams.  There is no CPU fallback: if the shared library is
+missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "librapid3.so")
+
+OK = 0
+ACT_SKIP, ACT_REUSE, ACT_ATTEND = 0, 1, 2
+
+EXPORTS = [
+    "rapid3_create", "rapid3_destroy", "rapid3_strerror", "rapid3_num_blocks", "rapid3_mask_words",
+    "rapid3_block_scores", "rapid3_select_mask", "rapid3_sparse_joint_attn", "rapid3_gated_step",
+    "rapid3_gated_step_host", "rapid3_workspace", "rapid3_launch_count", "rapid3_last_status",
+]
+
+
+class Rapid3Error(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [("B_max", ctypes.c_int32), ("H", ctypes.c_int32), ("D", ctypes.c_int32),
+                ("n_text", ctypes.c_int32), ("n_image", ctypes.c_int32), ("block", ctypes.c_int32),
+                ("stride_b", ctypes.c_int64), ("stride_h", ctypes.c_int64), ("stride_n", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads librapid3.so (built in-tree by paper_2509_22323_b200.build); raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} not found: build the CUDA library first (python -m paper_2509_22323_b200.build); "
+            "there is no CPU fallback")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+    i32p, f32p, i64p = ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int64)
+    lib.rapid3_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Shape)]
+    lib.rapid3_destroy.argtypes = [vp]
+    lib.rapid3_strerror.argtypes = [ci]
+    lib.rapid3_strerror.restype = ctypes.c_char_p
+    lib.rapid3_num_blocks.argtypes = [ctypes.POINTER(Shape)]
+    lib.rapid3_mask_words.argtypes = [ctypes.POINTER(Shape)]
+    lib.rapid3_block_scores.argtypes = [vp, vp, vp, i32p, ci, vp, vp]
+    lib.rapid3_select_mask.argtypes = [vp, vp, f32p, ci, vp, vp, vp, vp]
+    lib.rapid3_sparse_joint_attn.argtypes = [vp, vp, vp, vp, vp, i32p, ci, vp, vp, cf, vp]
+    lib.rapid3_gated_step.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp]
+    lib.rapid3_gated_step_host.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp, i64p, i64p]
+    lib.rapid3_workspace.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
+    lib.rapid3_launch_count.argtypes = [vp]
+    lib.rapid3_launch_count.restype = ctypes.c_int64
+    lib.rapid3_last_status.argtypes = [vp, ctypes.POINTER(ci)]
+    _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load().rapid3_strerror(int(code)).decode()
+
+
+def _check(code: int, what: str):
+    if code != OK:
+        raise Rapid3Error(code, what)
+
+
+def _i32(xs: Optional[Sequence[int]]):
+    if xs is None:
+        return None
+    return (ctypes.c_int32 * len(xs))(*[int(x) for x in xs])
+
+
+def _f32(xs: Sequence[float]):
+    return (ctypes.c_float * len(xs))(*[float(x) for x in xs])
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+class Context:
+    """Owns a rapid3_ctx for tensors of shape [B<=B_max, H, N, D] with the given element strides."""
+
+    def __init__(self, B_max: int, H: int, D: int, n_text: int, n_image: int,
+                 strides: Optional[Sequence[int]] = None):
+        self.lib = load()
+        N = n_text + n_image
+        if strides is None:
+            strides = (H * N * D, N * D, D)
+        self.shape = Shape(B_max, H, D, n_text, n_image, 64, int(strides[0]), int(strides[1]), int(strides[2]))
+        self.B_max, self.H, self.D, self.n_text, self.n_image, self.N = B_max, H, D, n_text, n_image, N
+        self.handle = ctypes.c_void_p()
+        _check(self.lib.rapid3_create(ctypes.byref(self.handle), ctypes.byref(self.shape)), "rapid3_create")
+        self.nb = self.lib.rapid3_num_blocks(ctypes.byref(self.shape))
+        self.words = self.lib.rapid3_mask_words(ctypes.byref(self.shape))
+
+    def close(self):
+        if getattr(self, "handle", None) is not None and self.handle.value:
+            self.lib.rapid3_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- the four calls of the path (same names as the C ABI) ----
+    def rapid3_block_scores(self, q: torch.Tensor, k: torch.Tensor, img_idx: Optional[Sequence[int]] = None,
+                            n_img: Optional[int] = None, scores: Optional[torch.Tensor] = None) -> torch.Tensor:
+        n = len(img_idx) if img_idx is not None else (n_img if n_img is not None else q.shape[0])
+        if scores is None:
+            scores = torch.empty((n, self.H, self.nb, self.nb), dtype=torch.float32, device=q.device)
+        _check(self.lib.rapid3_block_scores(self.handle, _ptr(q), _ptr(k), _i32(img_idx), n, _ptr(scores), _stream()),
+               "rapid3_block_scores")
+        return scores
+
+    def rapid3_select_mask(self, scores: torch.Tensor, keep_ratio: Sequence[float], out=None):
+        n = len(keep_ratio)
+        dev = scores.device
+        if out is None:
+            bitmask = torch.empty((n, self.H, self.nb, self.words), dtype=torch.int64, device=dev)
+            kept_idx = torch.empty((n, self.H, self.nb, self.nb), dtype=torch.int32, device=dev)
+            kept_cnt = torch.empty((n, self.H, self.nb), dtype=torch.int32, device=dev)
+        else:
+            bitmask, kept_idx, kept_cnt = out
+        _check(self.lib.rapid3_select_mask(self.handle, _ptr(scores), _f32(keep_ratio), n, _ptr(bitmask),
+                                           _ptr(kept_idx), _ptr(kept_cnt), _stream()), "rapid3_select_mask")
+        return bitmask, kept_idx, kept_cnt
+
+    def rapid3_sparse_joint_attn(self, q, k, v, out, img_idx: Optional[Sequence[int]] = None,
+                                 n_img: Optional[int] = None, kept_idx=None, kept_cnt=None,
+                                 softmax_scale: Optional[float] = None):
+        n = len(img_idx) if img_idx is not None else (n_img if n_img is not None else q.shape[0])
+        scale = softmax_scale if softmax_scale is not None else self.D ** -0.5
+        _check(self.lib.rapid3_sparse_joint_attn(self.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _i32(img_idx), n,
+                                                 _ptr(kept_idx), _ptr(kept_cnt), scale, _stream()),
+               "rapid3_sparse_joint_attn")
+        return out
+
+    def rapid3_gated_step(self, q, k, v, out, actions: Sequence[int], keep_ratio: Sequence[float],
+                          softmax_scale: Optional[float] = None):
+        scale = softmax_scale if softmax_scale is not None else self.D ** -0.5
+        _check(self.lib.rapid3_gated_step(self.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _i32(actions),
+                                          _f32(keep_ratio), len(actions), scale, _stream()), "rapid3_gated_step")
+        return out
+
+    def rapid3_gated_step_host(self, q, k, v, out, actions: Sequence[int], keep_ratio: Sequence[float],
+                               softmax_scale: Optional[float] = None):
+        """q, k, v, out: contiguous HOST bf16 tensors [B, H, N, D] (pinned for asynchronous copies)."""
+        scale = softmax_scale if softmax_scale is not None else self.D ** -0.5
+        up, down = ctypes.c_int64(0), ctypes.c_int64(0)
+        _check(self.lib.rapid3_gated_step_host(self.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _i32(actions),
+                                               _f32(keep_ratio), len(actions), scale, _stream(),
+                                               ctypes.byref(up), ctypes.byref(down)), "rapid3_gated_step_host")
+        return up.value, down.value
+
+    # ---- helpers ----
+    def workspace(self, n_sparse: int, device="cuda"):
+        """Views (no copy) of the scores / bitmask / kept lists the last gated step wrote."""
+        ptrs = [ctypes.c_void_p() for _ in range(4)]
+        _check(self.lib.rapid3_workspace(self.handle, *[ctypes.byref(p) for p in ptrs]), "rapid3_workspace")
+        shapes = [((n_sparse, self.H, self.nb, self.nb), torch.float32),
+                  ((n_sparse, self.H, self.nb, self.words), torch.int64),
+                  ((n_sparse, self.H, self.nb, self.nb), torch.int32),
+                  ((n_sparse, self.H, self.nb), torch.int32)]
+        return [_view(p.value, s, d, device) for p, (s, d) in zip(ptrs, shapes)]
+
+    def launch_count(self) -> int:
+        return int(self.lib.rapid3_launch_count(self.handle))
+
+    def last_status(self) -> int:
+        v = ctypes.c_int(0)
+        _check(self.lib.rapid3_last_status(self.handle, ctypes.byref(v)), "rapid3_last_status")
+        return v.value
+
+
+class _Raw:
+    """Minimal __cuda_array_interface__ carrier so torch can view library-owned device memory."""
+
+    def __init__(self, ptr, shape, typestr):
+        self.__cuda_array_interface__ = {"shape": tuple(shape), "typestr": typestr, "data": (ptr, False), "version": 2}
+
+
+def _view(ptr: int, shape, dtype, device):
+    typestr = {torch.float32: "<f4", torch.int64: "<i8", torch.int32: "<i4"}[dtype]
+    return torch.as_tensor(_Raw(ptr, shape, typestr), device=device)
+
+
+def bitmask_to_dense(bitmask: torch.Tensor, nb: int) -> torch.Tensor:
+    """[..., nb, words] int64 bitmask -> [..., nb, nb] uint8 (marshalling for tests and reports)."""
+    bm = bitmask.cpu()
+    j = torch.arange(nb)
+    words = bm[..., (j // 64)]
+    return ((words >> (j % 64)) & 1).to(torch.uint8)

@@ -1,0 +1,370 @@
+// Host side of the C ABI declared in rapid3.h: argument checks, workspace, tensor-map
+// construction (cuTensorMapEncodeTiled through the runtime's driver entry point), the gate /
+// compaction of rapid3_gated_step, and the kernel launches.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+
+#include "common.cuh"
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct MapSlot {
+    const void* ptr = nullptr;
+    CUtensorMap map;
+};
+
+}  // namespace
+
+struct rapid3_ctx {
+    rapid3_shape shape;
+    TensorGeom g;
+    int words;                    // uint64 words per bitmask row
+    // workspace (device)
+    double* pooled = nullptr;     // [2][B_max][H][nb][D]
+    float* scores = nullptr;      // [B_max][H][nb][nb]
+    uint64_t* bitmask = nullptr;  // [B_max][H][nb][words]
+    int32_t* kept_idx = nullptr;  // [B_max][H][nb][nb]
+    int32_t* kept_cnt = nullptr;  // [B_max][H][nb]
+    int* status = nullptr;
+    // host-tensor staging of rapid3_gated_step_host (created on first use)
+    void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
+    EncodeTiledFn encode = nullptr;
+    MapSlot maps[6];              // small cache keyed by base pointer
+    int map_rr = 0;
+    int64_t launches = 0;
+};
+
+namespace {
+
+int keep_count(double ratio, int n_free) {
+    double x = ceil(ratio * (double)n_free - 1e-6);
+    if (x < 0) x = 0;
+    if (x > n_free) x = n_free;
+    return (int)x;
+}
+
+int check_shape(const rapid3_shape* s) {
+    if (!s) return RAPID3_ERR_INVALID_ARG;
+    if (s->block != 64) return RAPID3_ERR_UNSUPPORTED;
+    if (s->D != 64 && s->D != 128) return RAPID3_ERR_UNSUPPORTED;
+    if (s->B_max < 1 || s->B_max > RAPID3_MAX_IMG || s->H < 1 || s->H > 65535) return RAPID3_ERR_INVALID_ARG;
+    if (s->n_text < 0 || s->n_image < 0) return RAPID3_ERR_INVALID_ARG;
+    long long N = (long long)s->n_text + s->n_image;
+    if (N < 1) return RAPID3_ERR_INVALID_ARG;
+    if (N > 64ll * RAPID3_MAX_NB) return RAPID3_ERR_UNSUPPORTED;
+    if (s->stride_n < s->D || s->stride_h < 1 || s->stride_b < 1) return RAPID3_ERR_INVALID_ARG;
+    if ((s->stride_n % 8) || (s->stride_h % 8) || (s->stride_b % 8)) return RAPID3_ERR_INVALID_ARG;
+    return RAPID3_OK;
+}
+
+int build_list(const rapid3_ctx* c, const int32_t* img_idx_host, int n_img, ImgList* l) {
+    if (n_img < 1 || n_img > c->shape.B_max) return RAPID3_ERR_INVALID_ARG;
+    l->n = n_img;
+    for (int p = 0; p < n_img; ++p) {
+        int b = img_idx_host ? img_idx_host[p] : p;
+        if (b < 0 || b >= c->shape.B_max) return RAPID3_ERR_INVALID_ARG;
+        l->batch[p] = b;
+        l->slot[p] = p;
+        l->k_free[p] = 0;
+    }
+    return RAPID3_OK;
+}
+
+// Tensor map over a bf16 [B, H, N, D] tensor: box = 64 channels x 64 tokens, 128-byte swizzle,
+// out-of-range tokens read as zero.
+int get_map(rapid3_ctx* c, const void* base, const CUtensorMap** out) {
+    for (auto& m : c->maps)
+        if (m.ptr == base) { *out = &m.map; return RAPID3_OK; }
+    if (reinterpret_cast<uintptr_t>(base) % 16) return RAPID3_ERR_INVALID_ARG;
+    MapSlot& m = c->maps[c->map_rr];
+    c->map_rr = (c->map_rr + 1) % 6;
+    const rapid3_shape& s = c->shape;
+    cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)c->g.N, (cuuint64_t)s.H, (cuuint64_t)s.B_max};
+    cuuint64_t strides[3] = {(cuuint64_t)s.stride_n * 2, (cuuint64_t)s.stride_h * 2, (cuuint64_t)s.stride_b * 2};
+    cuuint32_t box[4] = {64, 64, 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = c->encode(&m.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+                           estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { m.ptr = nullptr; return RAPID3_ERR_CUDA; }
+    m.ptr = base;
+    *out = &m.map;
+    return RAPID3_OK;
+}
+
+int attn_launch(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out, const ImgList& l,
+                const int32_t* kept_idx, const int32_t* kept_cnt, float scale, cudaStream_t st) {
+    const CUtensorMap *mq, *mk, *mv;
+    int r;
+    if ((r = get_map(c, q, &mq)) || (r = get_map(c, k, &mk)) || (r = get_map(c, v, &mv))) return r;
+    if (reinterpret_cast<uintptr_t>(out) % 16) return RAPID3_ERR_INVALID_ARG;
+    CUtensorMap tq = *mq, tk = *mk, tv = *mv;   // copies: a later get_map may recycle the slot
+    if (launch_attention(tq, tk, tv, out, c->g, l, kept_idx, kept_cnt, scale, c->status, st) != cudaSuccess)
+        return RAPID3_ERR_CUDA;
+    c->launches += 1;
+    return RAPID3_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* rapid3_strerror(int code) {
+    switch (code) {
+        case RAPID3_OK: return "ok";
+        case RAPID3_ERR_INVALID_ARG: return "invalid argument";
+        case RAPID3_ERR_UNSUPPORTED: return "unsupported shape";
+        case RAPID3_ERR_WORKSPACE: return "workspace allocation failed or size limit exceeded";
+        case RAPID3_ERR_CUDA: return "CUDA call failed";
+        case RAPID3_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case RAPID3_ERR_BAD_LIST: return "kept-list entry out of range";
+        default: return "unknown status";
+    }
+}
+
+int rapid3_num_blocks(const rapid3_shape* s) {
+    if (check_shape(s) != RAPID3_OK) return check_shape(s);
+    return (int)(((long long)s->n_text + s->n_image + 63) / 64);
+}
+
+int rapid3_mask_words(const rapid3_shape* s) {
+    int nb = rapid3_num_blocks(s);
+    return nb < 0 ? nb : (nb + 63) / 64;
+}
+
+int rapid3_create(rapid3_ctx** out, const rapid3_shape* shape) {
+    if (!out) return RAPID3_ERR_INVALID_ARG;
+    *out = nullptr;
+    int r = check_shape(shape);
+    if (r != RAPID3_OK) return r;
+    rapid3_ctx* c = new (std::nothrow) rapid3_ctx();
+    if (!c) return RAPID3_ERR_WORKSPACE;
+    c->shape = *shape;
+    TensorGeom& g = c->g;
+    g.H = shape->H;
+    g.D = shape->D;
+    g.N = shape->n_text + shape->n_image;
+    g.nb = (g.N + 63) / 64;
+    g.n_text_blocks = (shape->n_text + 63) / 64;
+    g.stride_b = shape->stride_b;
+    g.stride_h = shape->stride_h;
+    g.stride_n = shape->stride_n;
+    c->words = (g.nb + 63) / 64;
+
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess) {
+        delete c;
+        return RAPID3_ERR_CUDA;
+    }
+    c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+
+    const size_t B = shape->B_max, H = g.H, nb = g.nb;
+    bool ok = cudaMalloc(&c->pooled, 2 * B * H * nb * g.D * sizeof(double)) == cudaSuccess &&
+              cudaMalloc(&c->scores, B * H * nb * nb * sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&c->bitmask, B * H * nb * c->words * sizeof(uint64_t)) == cudaSuccess &&
+              cudaMalloc(&c->kept_idx, B * H * nb * nb * sizeof(int32_t)) == cudaSuccess &&
+              cudaMalloc(&c->kept_cnt, B * H * nb * sizeof(int32_t)) == cudaSuccess &&
+              cudaMalloc(&c->status, sizeof(int)) == cudaSuccess &&
+              cudaMemset(c->status, 0, sizeof(int)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        rapid3_destroy(c);
+        return RAPID3_ERR_WORKSPACE;
+    }
+    if (attention_static_init() != cudaSuccess) {
+        cudaGetLastError();
+        rapid3_destroy(c);
+        return RAPID3_ERR_CUDA;
+    }
+    *out = c;
+    return RAPID3_OK;
+}
+
+int rapid3_destroy(rapid3_ctx* c) {
+    if (!c) return RAPID3_ERR_INVALID_ARG;
+    cudaFree(c->pooled);
+    cudaFree(c->scores);
+    cudaFree(c->bitmask);
+    cudaFree(c->kept_idx);
+    cudaFree(c->kept_cnt);
+    cudaFree(c->status);
+    for (void* s : c->stage) cudaFree(s);
+    delete c;
+    return RAPID3_OK;
+}
+
+int rapid3_block_scores(rapid3_ctx* c, const void* q, const void* k, const int32_t* img_idx_host, int n_img,
+                        float* scores, void* stream) {
+    if (!c || !q || !k || !scores) return RAPID3_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q) % 16) || (reinterpret_cast<uintptr_t>(k) % 16)) return RAPID3_ERR_INVALID_ARG;
+    ImgList l;
+    int r = build_list(c, img_idx_host, n_img, &l);
+    if (r != RAPID3_OK) return r;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (launch_block_pool(q, k, c->g, l, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+    if (launch_block_scores(c->pooled, c->g, n_img, scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+    c->launches += 2;
+    return RAPID3_OK;
+}
+
+int rapid3_select_mask(rapid3_ctx* c, const float* scores, const float* keep_ratio_host, int n_img,
+                       uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, void* stream) {
+    if (!c || !scores || !keep_ratio_host || !bitmask || !kept_idx || !kept_cnt) return RAPID3_ERR_INVALID_ARG;
+    ImgList l;
+    int r = build_list(c, nullptr, n_img, &l);
+    if (r != RAPID3_OK) return r;
+    const int n_free_img = c->g.nb - c->g.n_text_blocks - 1;   // free candidates of an image query row
+    for (int p = 0; p < n_img; ++p) {
+        const float ratio = keep_ratio_host[p];
+        if (!(ratio > 0.f) || !(ratio <= 1.f)) return RAPID3_ERR_INVALID_ARG;
+        l.k_free[p] = keep_count((double)ratio, n_free_img > 0 ? n_free_img : 0);
+    }
+    if (launch_select_mask(scores, c->g, l, bitmask, kept_idx, kept_cnt, static_cast<cudaStream_t>(stream)) !=
+        cudaSuccess)
+        return RAPID3_ERR_CUDA;
+    c->launches += 1;
+    return RAPID3_OK;
+}
+
+int rapid3_sparse_joint_attn(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
+                             const int32_t* img_idx_host, int n_img, const int32_t* kept_idx,
+                             const int32_t* kept_cnt, float softmax_scale, void* stream) {
+    if (!c || !q || !k || !v || !out) return RAPID3_ERR_INVALID_ARG;
+    if ((kept_idx == nullptr) != (kept_cnt == nullptr)) return RAPID3_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return RAPID3_ERR_INVALID_ARG;
+    ImgList l;
+    int r = build_list(c, img_idx_host, n_img, &l);
+    if (r != RAPID3_OK) return r;
+    if (!kept_idx)
+        for (int p = 0; p < n_img; ++p) l.slot[p] = -1;
+    return attn_launch(c, q, k, v, out, l, kept_idx, kept_cnt, softmax_scale, static_cast<cudaStream_t>(stream));
+}
+
+int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
+                      const int32_t* action_host, const float* keep_ratio_host, int B, float softmax_scale,
+                      void* stream) {
+    if (!c || !q || !k || !v || !out || !action_host || !keep_ratio_host) return RAPID3_ERR_INVALID_ARG;
+    if (B < 1 || B > c->shape.B_max) return RAPID3_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return RAPID3_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int n_free_img = c->g.nb - c->g.n_text_blocks - 1;
+    // gate + compaction: sparse images (ascending batch order) get workspace slots 0..ns-1;
+    // the attention list puts dense images first (longest work first), then sparse by ratio
+    ImgList sparse, all;
+    sparse.n = 0;
+    all.n = 0;
+    float ratio_of[RAPID3_MAX_IMG];
+    for (int b = 0; b < B; ++b) {
+        const int a = action_host[b];
+        if (a != RAPID3_ACT_SKIP && a != RAPID3_ACT_REUSE && a != RAPID3_ACT_ATTEND) return RAPID3_ERR_INVALID_ARG;
+        if (a != RAPID3_ACT_ATTEND) continue;
+        const float ratio = keep_ratio_host[b];
+        if (!(ratio > 0.f) || !(ratio <= 1.f)) return RAPID3_ERR_INVALID_ARG;
+        int slot = -1;
+        if (ratio < 1.f) {
+            slot = sparse.n++;
+            sparse.batch[slot] = b;
+            sparse.slot[slot] = slot;
+            sparse.k_free[slot] = keep_count((double)ratio, n_free_img > 0 ? n_free_img : 0);
+        }
+        int pos = all.n++;
+        while (pos > 0 && ratio_of[pos - 1] < ratio) {   // insertion sort, descending ratio, stable
+            all.batch[pos] = all.batch[pos - 1];
+            all.slot[pos] = all.slot[pos - 1];
+            ratio_of[pos] = ratio_of[pos - 1];
+            --pos;
+        }
+        all.batch[pos] = b;
+        all.slot[pos] = slot;
+        all.k_free[pos] = 0;
+        ratio_of[pos] = ratio;
+    }
+    if (all.n == 0) return RAPID3_OK;                     // every image gated: nothing is launched
+    if (sparse.n > 0) {
+        if ((reinterpret_cast<uintptr_t>(q) % 16) || (reinterpret_cast<uintptr_t>(k) % 16)) return RAPID3_ERR_INVALID_ARG;
+        if (launch_block_pool(q, k, c->g, sparse, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+        if (launch_block_scores(c->pooled, c->g, sparse.n, c->scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+        if (launch_select_mask(c->scores, c->g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st) != cudaSuccess)
+            return RAPID3_ERR_CUDA;
+        c->launches += 3;
+    }
+    return attn_launch(c, q, k, v, out, all, sparse.n ? c->kept_idx : nullptr, sparse.n ? c->kept_cnt : nullptr,
+                       softmax_scale, st);
+}
+
+int rapid3_gated_step_host(rapid3_ctx* c, const void* q_host, const void* k_host, const void* v_host, void* out_host,
+                           const int32_t* action_host, const float* keep_ratio_host, int B, float softmax_scale,
+                           void* stream, int64_t* bytes_h2d, int64_t* bytes_d2h) {
+    if (!c || !q_host || !k_host || !v_host || !out_host || !action_host || !keep_ratio_host)
+        return RAPID3_ERR_INVALID_ARG;
+    if (B < 1 || B > c->shape.B_max) return RAPID3_ERR_INVALID_ARG;
+    const rapid3_shape& s = c->shape;
+    const long long N = c->g.N;
+    // staging is contiguous [B, H, N, D]; the context's strides must describe exactly that
+    if (s.stride_n != s.D || s.stride_h != N * s.D || s.stride_b != (long long)s.H * N * s.D)
+        return RAPID3_ERR_UNSUPPORTED;
+    const size_t img_bytes = (size_t)s.H * N * s.D * 2;
+    if (!c->stage[0]) {
+        for (int i = 0; i < 4; ++i)
+            if (cudaMalloc(&c->stage[i], img_bytes * s.B_max) != cudaSuccess) {
+                cudaGetLastError();
+                for (int j = 0; j < 4; ++j) { cudaFree(c->stage[j]); c->stage[j] = nullptr; }
+                return RAPID3_ERR_WORKSPACE;
+            }
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const void* src[3] = {q_host, k_host, v_host};
+    int64_t up = 0, down = 0;
+    for (int b = 0; b < B; ++b) {
+        if (action_host[b] != RAPID3_ACT_ATTEND) continue;
+        for (int i = 0; i < 3; ++i) {
+            if (cudaMemcpyAsync((char*)c->stage[i] + b * img_bytes, (const char*)src[i] + b * img_bytes, img_bytes,
+                                cudaMemcpyHostToDevice, st) != cudaSuccess)
+                return RAPID3_ERR_CUDA;
+            up += (int64_t)img_bytes;
+        }
+    }
+    int r = rapid3_gated_step(c, c->stage[0], c->stage[1], c->stage[2], c->stage[3], action_host, keep_ratio_host, B,
+                              softmax_scale, stream);
+    if (r != RAPID3_OK) return r;
+    for (int b = 0; b < B; ++b) {
+        if (action_host[b] != RAPID3_ACT_ATTEND) continue;
+        if (cudaMemcpyAsync((char*)out_host + b * img_bytes, (const char*)c->stage[3] + b * img_bytes, img_bytes,
+                            cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return RAPID3_ERR_CUDA;
+        down += (int64_t)img_bytes;
+    }
+    if (bytes_h2d) *bytes_h2d = up;
+    if (bytes_d2h) *bytes_d2h = down;
+    return RAPID3_OK;
+}
+
+int rapid3_workspace(rapid3_ctx* c, float** scores, uint64_t** bitmask, int32_t** kept_idx, int32_t** kept_cnt) {
+    if (!c) return RAPID3_ERR_INVALID_ARG;
+    if (scores) *scores = c->scores;
+    if (bitmask) *bitmask = c->bitmask;
+    if (kept_idx) *kept_idx = c->kept_idx;
+    if (kept_cnt) *kept_cnt = c->kept_cnt;
+    return RAPID3_OK;
+}
+
+int64_t rapid3_launch_count(rapid3_ctx* c) { return c ? c->launches : -1; }
+
+int rapid3_last_status(rapid3_ctx* c, int* device_status) {
+    if (!c || !device_status) return RAPID3_ERR_INVALID_ARG;
+    int v = 0;
+    if (cudaMemcpy(&v, c->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return RAPID3_ERR_CUDA;
+    if (v != 0 && cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess) return RAPID3_ERR_CUDA;
+    *device_status = v;
+    return RAPID3_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,42 @@
+// Shared declarations of the rapid3 CUDA library: launch-argument structs and the internal
+// launcher prototypes.  Host API in api.cu; kernels in k1_scores.cu, k2_select.cu, k3_attn.cu.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rapid3.h"
+
+#define RAPID3_BLOCK 64
+#define RAPID3_MAX_IMG 64     // images per launch (lists travel as kernel arguments)
+#define RAPID3_MAX_NB 1024    // key blocks per sequence (65536 tokens)
+
+// Per-launch image list.  batch[p]: index into the B dimension of Q/K/V/O.
+// slot[p]: index into the compacted scores / mask / kept-list arrays, or -1 for a dense image.
+// k_free[p]: free candidates kept per image row (select kernel).
+struct ImgList {
+    int n;
+    int batch[RAPID3_MAX_IMG];
+    int slot[RAPID3_MAX_IMG];
+    int k_free[RAPID3_MAX_IMG];
+};
+
+struct TensorGeom {
+    int H, D, N, nb, n_text_blocks;
+    long long stride_b, stride_h, stride_n;   // elements
+};
+
+// K1: block means of Q and K (fp64) for the listed images, then S = Qbar . Kbar^T -> fp32.
+cudaError_t launch_block_pool(const void* q, const void* k, const TensorGeom& g, const ImgList& imgs,
+                              double* pooled /* [2][n][H][nb][D] */, cudaStream_t s);
+cudaError_t launch_block_scores(const double* pooled, const TensorGeom& g, int n_img, float* scores,
+                                cudaStream_t s);
+// K2: forced + top-k selection.
+cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const ImgList& imgs,
+                               uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s);
+// K3: attention over kept tiles.
+cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv,
+                             void* out, const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
+                             const int32_t* kept_cnt, float softmax_scale, int* status, cudaStream_t s);
+cudaError_t attention_static_init();

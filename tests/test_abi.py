@@ -1,0 +1,36 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares."""
+import os
+import re
+
+from paper_2509_22323_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "rapid3.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rapid3_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = binding.load()
+    names = declared_symbols()
+    assert len(names) >= 12
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_strerror_and_shape_helpers_run_on_the_host():
+    assert binding.strerror(0) == "ok"
+    assert "wait" in binding.strerror(-5)
+    lib = binding.load()
+    import ctypes
+    s = binding.Shape(3, 24, 128, 512, 4096, 64, 24 * 4608 * 128, 4608 * 128, 128)
+    assert lib.rapid3_num_blocks(ctypes.byref(s)) == 72
+    assert lib.rapid3_mask_words(ctypes.byref(s)) == 2
+    s2 = binding.Shape(2, 24, 64, 333, 4096, 64, 24 * 4429 * 64, 4429 * 64, 64)
+    assert lib.rapid3_num_blocks(ctypes.byref(s2)) == 70
+    bad = binding.Shape(1, 2, 96, 64, 256, 64, 1, 1, 96)
+    assert lib.rapid3_num_blocks(ctypes.byref(bad)) == -2
