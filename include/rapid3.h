@@ -151,6 +151,16 @@ int rapid3_workspace(rapid3_ctx* ctx, float** scores, uint64_t** bitmask, int32_
 /* Number of kernels this context has launched so far (all entry points). */
 int64_t rapid3_launch_count(rapid3_ctx* ctx);
 
+/*
+ * Measurement aid (no counterpart in the paper): with profiling enabled every kernel launch of
+ * this context is bracketed by a CUDA event pair on the caller's stream (at most 16384 pairs
+ * between reads).  rapid3_profile_read waits for the recorded events, returns the summed device
+ * time in milliseconds and the launch count per kernel kind
+ * (0 block pool, 1 block scores, 2 mask select, 3 attention) and clears the record.
+ */
+int rapid3_profile(rapid3_ctx* ctx, int enable);
+int rapid3_profile_read(rapid3_ctx* ctx, double* ms /* [4] */, int64_t* launches /* [4] */);
+
 /* Copies the device status word to *device_status (RAPID3_OK or a negative code) and clears it.
  * Synchronises the device; call it after the stream has been synchronised. */
 int rapid3_last_status(rapid3_ctx* ctx, int* device_status);

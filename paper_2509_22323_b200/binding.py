@@ -22,6 +22,7 @@ EXPORTS = [
     "rapid3_create", "rapid3_destroy", "rapid3_strerror", "rapid3_num_blocks", "rapid3_mask_words",
     "rapid3_block_scores", "rapid3_select_mask", "rapid3_sparse_joint_attn", "rapid3_gated_step",
     "rapid3_gated_step_host", "rapid3_workspace", "rapid3_launch_count", "rapid3_last_status",
+    "rapid3_profile", "rapid3_profile_read",
 ]
 
 
@@ -67,6 +68,8 @@ def load() -> ctypes.CDLL:
     lib.rapid3_launch_count.argtypes = [vp]
     lib.rapid3_launch_count.restype = ctypes.c_int64
     lib.rapid3_last_status.argtypes = [vp, ctypes.POINTER(ci)]
+    lib.rapid3_profile.argtypes = [vp, ci]
+    lib.rapid3_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), i64p]
     _lib = lib
     return lib
 
@@ -188,6 +191,17 @@ class Context:
 
     def launch_count(self) -> int:
         return int(self.lib.rapid3_launch_count(self.handle))
+
+    def profile(self, enable: bool):
+        _check(self.lib.rapid3_profile(self.handle, int(bool(enable))), "rapid3_profile")
+
+    def profile_read(self):
+        """Summed device milliseconds and launch counts per kernel kind since the last read."""
+        ms = (ctypes.c_double * 4)()
+        n = (ctypes.c_int64 * 4)()
+        _check(self.lib.rapid3_profile_read(self.handle, ms, n), "rapid3_profile_read")
+        kinds = ("block_pool", "block_scores", "select_mask", "attention")
+        return {k: (ms[i], n[i]) for i, k in enumerate(kinds)}
 
     def last_status(self) -> int:
         v = ctypes.c_int(0)

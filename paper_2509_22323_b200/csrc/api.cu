@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 
@@ -17,6 +18,11 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct MapSlot {
     const void* ptr = nullptr;
     CUtensorMap map;
+};
+
+struct ProfRec {
+    cudaEvent_t a, b;
+    int kind;
 };
 
 }  // namespace
@@ -38,9 +44,38 @@ struct rapid3_ctx {
     MapSlot maps[6];              // small cache keyed by base pointer
     int map_rr = 0;
     int64_t launches = 0;
+    // optional per-kernel timing (rapid3_profile): event pairs around each launch
+    bool prof_on = false;
+    std::vector<ProfRec> prof;
+    size_t prof_used = 0;
 };
 
 namespace {
+
+enum { PROF_POOL = 0, PROF_SCORES, PROF_SELECT, PROF_ATTN };
+
+// Records an event pair around one launch when profiling is on.
+struct ProfScope {
+    rapid3_ctx* c;
+    cudaStream_t st;
+    ProfRec* rec = nullptr;
+    ProfScope(rapid3_ctx* ctx, int kind, cudaStream_t s) : c(ctx), st(s) {
+        if (!c->prof_on) return;
+        if (c->prof_used == c->prof.size()) {
+            if (c->prof.size() >= 16384) return;
+            ProfRec r;
+            if (cudaEventCreate(&r.a) != cudaSuccess) return;
+            if (cudaEventCreate(&r.b) != cudaSuccess) { cudaEventDestroy(r.a); return; }
+            c->prof.push_back(r);
+        }
+        rec = &c->prof[c->prof_used++];
+        rec->kind = kind;
+        cudaEventRecord(rec->a, st);
+    }
+    ~ProfScope() {
+        if (rec) cudaEventRecord(rec->b, st);
+    }
+};
 
 int keep_count(double ratio, int n_free) {
     double x = ceil(ratio * (double)n_free - 1e-6);
@@ -105,8 +140,11 @@ int attn_launch(rapid3_ctx* c, const void* q, const void* k, const void* v, void
     if ((r = get_map(c, q, &mq)) || (r = get_map(c, k, &mk)) || (r = get_map(c, v, &mv))) return r;
     if (reinterpret_cast<uintptr_t>(out) % 16) return RAPID3_ERR_INVALID_ARG;
     CUtensorMap tq = *mq, tk = *mk, tv = *mv;   // copies: a later get_map may recycle the slot
-    if (launch_attention(tq, tk, tv, out, c->g, l, kept_idx, kept_cnt, scale, c->status, st) != cudaSuccess)
-        return RAPID3_ERR_CUDA;
+    {
+        ProfScope ps(c, PROF_ATTN, st);
+        if (launch_attention(tq, tk, tv, out, c->g, l, kept_idx, kept_cnt, scale, c->status, st) != cudaSuccess)
+            return RAPID3_ERR_CUDA;
+    }
     c->launches += 1;
     return RAPID3_OK;
 }
@@ -197,6 +235,7 @@ int rapid3_destroy(rapid3_ctx* c) {
     cudaFree(c->kept_cnt);
     cudaFree(c->status);
     for (void* s : c->stage) cudaFree(s);
+    for (auto& r : c->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     delete c;
     return RAPID3_OK;
 }
@@ -209,8 +248,14 @@ int rapid3_block_scores(rapid3_ctx* c, const void* q, const void* k, const int32
     int r = build_list(c, img_idx_host, n_img, &l);
     if (r != RAPID3_OK) return r;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (launch_block_pool(q, k, c->g, l, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
-    if (launch_block_scores(c->pooled, c->g, n_img, scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+    {
+        ProfScope ps(c, PROF_POOL, st);
+        if (launch_block_pool(q, k, c->g, l, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+    }
+    {
+        ProfScope ps(c, PROF_SCORES, st);
+        if (launch_block_scores(c->pooled, c->g, n_img, scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+    }
     c->launches += 2;
     return RAPID3_OK;
 }
@@ -227,9 +272,12 @@ int rapid3_select_mask(rapid3_ctx* c, const float* scores, const float* keep_rat
         if (!(ratio > 0.f) || !(ratio <= 1.f)) return RAPID3_ERR_INVALID_ARG;
         l.k_free[p] = keep_count((double)ratio, n_free_img > 0 ? n_free_img : 0);
     }
-    if (launch_select_mask(scores, c->g, l, bitmask, kept_idx, kept_cnt, static_cast<cudaStream_t>(stream)) !=
-        cudaSuccess)
-        return RAPID3_ERR_CUDA;
+    {
+        ProfScope ps(c, PROF_SELECT, static_cast<cudaStream_t>(stream));
+        if (launch_select_mask(scores, c->g, l, bitmask, kept_idx, kept_cnt, static_cast<cudaStream_t>(stream)) !=
+            cudaSuccess)
+            return RAPID3_ERR_CUDA;
+    }
     c->launches += 1;
     return RAPID3_OK;
 }
@@ -290,10 +338,19 @@ int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v
     if (all.n == 0) return RAPID3_OK;                     // every image gated: nothing is launched
     if (sparse.n > 0) {
         if ((reinterpret_cast<uintptr_t>(q) % 16) || (reinterpret_cast<uintptr_t>(k) % 16)) return RAPID3_ERR_INVALID_ARG;
-        if (launch_block_pool(q, k, c->g, sparse, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
-        if (launch_block_scores(c->pooled, c->g, sparse.n, c->scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
-        if (launch_select_mask(c->scores, c->g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st) != cudaSuccess)
-            return RAPID3_ERR_CUDA;
+        {
+            ProfScope ps(c, PROF_POOL, st);
+            if (launch_block_pool(q, k, c->g, sparse, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+        }
+        {
+            ProfScope ps(c, PROF_SCORES, st);
+            if (launch_block_scores(c->pooled, c->g, sparse.n, c->scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+        }
+        {
+            ProfScope ps(c, PROF_SELECT, st);
+            if (launch_select_mask(c->scores, c->g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st) != cudaSuccess)
+                return RAPID3_ERR_CUDA;
+        }
         c->launches += 3;
     }
     return attn_launch(c, q, k, v, out, all, sparse.n ? c->kept_idx : nullptr, sparse.n ? c->kept_cnt : nullptr,
@@ -357,6 +414,27 @@ int rapid3_workspace(rapid3_ctx* c, float** scores, uint64_t** bitmask, int32_t*
 }
 
 int64_t rapid3_launch_count(rapid3_ctx* c) { return c ? c->launches : -1; }
+
+int rapid3_profile(rapid3_ctx* c, int enable) {
+    if (!c) return RAPID3_ERR_INVALID_ARG;
+    c->prof_on = enable != 0;
+    return RAPID3_OK;
+}
+
+int rapid3_profile_read(rapid3_ctx* c, double* ms, int64_t* launches) {
+    if (!c || !ms || !launches) return RAPID3_ERR_INVALID_ARG;
+    for (int i = 0; i < 4; ++i) { ms[i] = 0.0; launches[i] = 0; }
+    for (size_t i = 0; i < c->prof_used; ++i) {
+        ProfRec& r = c->prof[i];
+        float t = 0.f;
+        if (cudaEventSynchronize(r.b) != cudaSuccess || cudaEventElapsedTime(&t, r.a, r.b) != cudaSuccess)
+            return RAPID3_ERR_CUDA;
+        ms[r.kind] += (double)t;
+        launches[r.kind] += 1;
+    }
+    c->prof_used = 0;
+    return RAPID3_OK;
+}
 
 int rapid3_last_status(rapid3_ctx* c, int* device_status) {
     if (!c || !device_status) return RAPID3_ERR_INVALID_ARG;
