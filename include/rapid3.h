@@ -161,6 +161,34 @@ int64_t rapid3_launch_count(rapid3_ctx* ctx);
 int rapid3_profile(rapid3_ctx* ctx, int enable);
 int rapid3_profile_read(rapid3_ctx* ctx, double* ms /* [4] */, int64_t* launches /* [4] */);
 
+/*
+ * Scoring pass without any allocation (the paper has no counterpart; this exists for the callers
+ * described here).  rapid3_create obtains the workspace with cudaMalloc.  Some hosts of this
+ * library cannot do that: an inference server whose own allocator has already reserved all of
+ * the GPU's memory (a later cudaMalloc from a plug-in fails), or a latency-critical sampling loop
+ * that must not take the device-wide synchronisation an allocation implies.  For them this
+ * entry point computes exactly what rapid3_block_scores computes -- scores[p][h][i][j], fp32,
+ * [n_img, H, nb, nb], same kernels, same rounding -- without a context: the block means go to a
+ * fixed array inside the library's device image instead of an allocated workspace.
+ *
+ *   - `shape` describes Q and K as for rapid3_create (B_max only bounds the batch indices).
+ *   - Limit: 2 * n_img * H * nb * D block means (fp64) must fit rapid3_static_scratch_bytes()
+ *     = 16 MiB, e.g. four FLUX 1024^2 images (24 heads, D = 128, 72 blocks) or one FLUX 2048^2
+ *     image per call; a larger request returns RAPID3_ERR_WORKSPACE and launches nothing.
+ *     Every GPU that loads the library holds these 16 MiB until the process exits.
+ *   - The first call on a device looks up the array's device address (once per device, with
+ *     that device current); make that first call before starting any stream capture.
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine; asynchronous on `stream`.
+ *   - All calls on a device share the one array and it keeps the previous call's contents.
+ *     Nothing in it has to start at zero (the pooling kernel writes every element the scoring
+ *     kernel reads), but two calls that overlap on the GPU (different streams, no dependency)
+ *     race on it: order them on one stream or with events.
+ */
+int rapid3_block_scores_static(const rapid3_shape* shape, const void* q, const void* k,
+                               const int32_t* img_idx_host, int n_img, float* scores, void* stream);
+/* Size in bytes of the fixed scratch array of rapid3_block_scores_static. */
+int64_t rapid3_static_scratch_bytes(void);
+
 /* Copies the device status word to *device_status (RAPID3_OK or a negative code) and clears it.
  * Synchronises the device; call it after the stream has been synchronised. */
 int rapid3_last_status(rapid3_ctx* ctx, int* device_status);

@@ -22,7 +22,7 @@ EXPORTS = [
     "rapid3_create", "rapid3_destroy", "rapid3_strerror", "rapid3_num_blocks", "rapid3_mask_words",
     "rapid3_block_scores", "rapid3_select_mask", "rapid3_sparse_joint_attn", "rapid3_gated_step",
     "rapid3_gated_step_host", "rapid3_workspace", "rapid3_launch_count", "rapid3_last_status",
-    "rapid3_profile", "rapid3_profile_read",
+    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes",
 ]
 
 
@@ -70,6 +70,9 @@ def load() -> ctypes.CDLL:
     lib.rapid3_last_status.argtypes = [vp, ctypes.POINTER(ci)]
     lib.rapid3_profile.argtypes = [vp, ci]
     lib.rapid3_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), i64p]
+    lib.rapid3_block_scores_static.argtypes = [ctypes.POINTER(Shape), vp, vp, i32p, ci, vp, vp]
+    lib.rapid3_static_scratch_bytes.argtypes = []
+    lib.rapid3_static_scratch_bytes.restype = ctypes.c_int64
     _lib = lib
     return lib
 
@@ -207,6 +210,21 @@ class Context:
         v = ctypes.c_int(0)
         _check(self.lib.rapid3_last_status(self.handle, ctypes.byref(v)), "rapid3_last_status")
         return v.value
+
+
+def rapid3_block_scores_static(shape: Shape, q: torch.Tensor, k: torch.Tensor, scores: torch.Tensor,
+                               img_idx: Optional[Sequence[int]] = None, n_img: Optional[int] = None) -> torch.Tensor:
+    """Context-free scoring pass for hosts that may not allocate device memory: the block means go
+    to the fixed array inside the library instead of a workspace.  `scores` ([n, H, nb, nb] fp32,
+    device) is supplied by the caller; nothing is allocated here either."""
+    n = len(img_idx) if img_idx is not None else (n_img if n_img is not None else q.shape[0])
+    _check(load().rapid3_block_scores_static(ctypes.byref(shape), _ptr(q), _ptr(k), _i32(img_idx), n, _ptr(scores),
+                                             _stream()), "rapid3_block_scores_static")
+    return scores
+
+
+def static_scratch_bytes() -> int:
+    return int(load().rapid3_static_scratch_bytes())
 
 
 class _Raw:

@@ -107,3 +107,92 @@ cudaError_t launch_block_scores(const double* pooled, const TensorGeom& g, int n
     scores_kernel<<<grid, 256, 0, s>>>(pooled, g, n_img, scores);
     return cudaGetLastError();
 }
+
+// ---------------------------------------------------------------------------------------------
+// rapid3_block_scores_static: the scoring pass for callers that may not allocate device memory.
+//
+// The block means (the only scratch of this pass) live in the file-scope array below instead of
+// a cudaMalloc'ed workspace.  The array is part of the loaded module: every GPU that loads the
+// library holds RAPID3_STATIC_SCRATCH_DOUBLES * 8 bytes (16 MiB) until the process exits.
+// In host code the array's name is only a stand-in for the symbol, not a device address, so the
+// address is looked up once per device with cudaGetSymbolAddress (with that device current) and
+// that pointer is what the kernels get.
+#include <mutex>
+
+#define RAPID3_STATIC_SCRATCH_DOUBLES (1ll << 21)   // 16 MiB of fp64 block means
+static __device__ __align__(256) double g_static_pool_scratch[RAPID3_STATIC_SCRATCH_DOUBLES];
+
+namespace {
+
+constexpr int RAPID3_STATIC_MAX_DEVICES = 64;
+
+std::mutex g_static_mu;
+double* g_static_ptr[RAPID3_STATIC_MAX_DEVICES] = {};
+
+// Device address of the scratch array on the current device (looked up on first use per device).
+int static_scratch(double** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= RAPID3_STATIC_MAX_DEVICES) return RAPID3_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_pool_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return RAPID3_ERR_CUDA;
+        }
+        g_static_ptr[dev] = static_cast<double*>(p);
+    }
+    *out = g_static_ptr[dev];
+    return RAPID3_OK;
+}
+
+}  // namespace
+
+extern "C" int rapid3_block_scores_static(const rapid3_shape* s, const void* q, const void* k,
+                                          const int32_t* img_idx_host, int n_img, float* scores, void* stream) {
+    if (!s || !q || !k || !scores) return RAPID3_ERR_INVALID_ARG;
+    if (s->block != RAPID3_BLOCK || (s->D != 64 && s->D != 128)) return RAPID3_ERR_UNSUPPORTED;
+    if (s->B_max < 1 || s->B_max > RAPID3_MAX_IMG || s->H < 1 || s->H > 65535) return RAPID3_ERR_INVALID_ARG;
+    if (s->n_text < 0 || s->n_image < 0) return RAPID3_ERR_INVALID_ARG;
+    const long long N = (long long)s->n_text + s->n_image;
+    if (N < 1) return RAPID3_ERR_INVALID_ARG;
+    if (N > 64ll * RAPID3_MAX_NB) return RAPID3_ERR_UNSUPPORTED;
+    if (s->stride_n < s->D || s->stride_h < 1 || s->stride_b < 1) return RAPID3_ERR_INVALID_ARG;
+    if ((s->stride_n % 8) || (s->stride_h % 8) || (s->stride_b % 8)) return RAPID3_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q) % 16) || (reinterpret_cast<uintptr_t>(k) % 16)) return RAPID3_ERR_INVALID_ARG;
+    if (n_img < 1 || n_img > s->B_max) return RAPID3_ERR_INVALID_ARG;
+
+    TensorGeom g;
+    g.H = s->H;
+    g.D = s->D;
+    g.N = (int)N;
+    g.nb = (int)((N + 63) / 64);
+    g.n_text_blocks = (s->n_text + 63) / 64;
+    g.stride_b = s->stride_b;
+    g.stride_h = s->stride_h;
+    g.stride_n = s->stride_n;
+    // block means of Q and K for the listed images must fit the fixed array
+    const long long need = 2ll * n_img * g.H * g.nb * g.D;
+    if (need > RAPID3_STATIC_SCRATCH_DOUBLES) return RAPID3_ERR_WORKSPACE;
+
+    ImgList l;
+    l.n = n_img;
+    for (int p = 0; p < n_img; ++p) {
+        const int b = img_idx_host ? img_idx_host[p] : p;
+        if (b < 0 || b >= s->B_max) return RAPID3_ERR_INVALID_ARG;
+        l.batch[p] = b;
+        l.slot[p] = p;
+        l.k_free[p] = 0;
+    }
+    double* scratch = nullptr;
+    const int r = static_scratch(&scratch);
+    if (r != RAPID3_OK) return r;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // every element of the used part of the scratch is written by the pooling kernel before the
+    // scoring kernel reads it, so nothing has to be cleared between calls
+    if (launch_block_pool(q, k, g, l, scratch, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+    if (launch_block_scores(scratch, g, n_img, scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+    return RAPID3_OK;
+}
+
+extern "C" int64_t rapid3_static_scratch_bytes(void) { return RAPID3_STATIC_SCRATCH_DOUBLES * (int64_t)sizeof(double); }
