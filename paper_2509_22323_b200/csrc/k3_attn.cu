@@ -1,21 +1,23 @@
 // K3: masked flash-style joint attention over the kept key tiles (sm_100a).
 //
 // One CTA per (image, head, pair of adjacent 64-token query blocks) = a 128-row Q tile, the
-// native UMMA M.  The two query blocks' ascending kept lists are merged into one union list;
-// the CTA walks it two key blocks (128 keys) at a time.  A 64x64 sub-tile whose key block is
-// not in that query block's own list is masked out before the softmax, so each query block
-// attends exactly its own kept set.
+// native UMMA M.  The two query blocks' ascending kept lists are merged into one union list and
+// the CTA walks it one 64-token key block at a time.  A 64x64 sub-tile whose key block is not
+// in that query block's own list gets P = 0, so each query block attends exactly its own kept
+// set.
 //
-// Roles (192 threads):
-//   warps 0-3  softmax: thread = one query row; S from TMEM (tcgen05.ld), fp32 online softmax
-//              with lazy rescale, P written back to TMEM as bf16 (aliasing S), final O / l store
-//   warp 4     producer: TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of Q once and of
-//              gathered K / V key blocks per tile
-//   warp 5     TMEM allocation and UMMA issue: S = Q K^T (both operands in shared memory),
-//              O += P V (P from TMEM, V from shared memory as an N-major operand)
-// Two CTAs are resident per SM (2 x 256 TMEM columns, ~100 KB shared memory each) so one CTA's
-// softmax overlaps the other's MMAs.  Every mbarrier wait is bounded; a wait that runs out
-// records RAPID3_ERR_TIMEOUT in the status word and the CTA drains and exits normally.
+// Pipeline inside a CTA (192 threads):
+//   warp 4     producer: TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of Q once, then the
+//              gathered K and V blocks into two rings of shared-memory stages
+//   warp 5     TMEM allocation and UMMA issue.  S is double buffered in TMEM (2 x 64 fp32
+//              columns): S(j+1) = Q K(j+1)^T is issued before O += P(j) V(j), so the tensor pipe
+//              works on the next scores while the softmax warps are busy with the current ones
+//   warps 0-3  softmax: thread = one query row; S(j) from TMEM in one pass (64 registers), fp32
+//              online softmax with lazy rescale of O, P(j) written back over S(j) as bf16,
+//              final O / l store
+// Two CTAs are resident per SM (2 x 256 TMEM columns, ~100 KB shared memory each).
+// Every mbarrier wait is bounded; a wait that runs out records RAPID3_ERR_TIMEOUT in the status
+// word and the CTA drains its copies, releases its TMEM and exits normally.
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -25,11 +27,12 @@ namespace {
 
 constexpr int NTHREADS = 192;
 constexpr int TMEM_COLS = 256;
-constexpr int S_COL = 0;
+constexpr int S_COL = 0;            // S(j) at columns [64 * (j & 1), +64); P(j) over its first 32
 constexpr int O_COL = 128;
-constexpr int HALF_BYTES = 16384;   // one 64-channel half of a 128-row tile: 128 rows x 128 bytes
-constexpr int BLK_BYTES = 8192;     // 64 rows x 128 bytes
+constexpr int BLK_BYTES = 8192;     // 64 rows x 128 bytes: one 64-channel half of a 64-token block
+constexpr int QHALF_BYTES = 16384;  // one 64-channel half of the 128-row Q tile
 constexpr float RESCALE_LOG2 = 8.0f;
+constexpr int MAX_STAGES = 4;
 
 struct AttnParams {
     TensorGeom g;
@@ -41,10 +44,22 @@ struct AttnParams {
     float scale_log2;
 };
 
-enum { BAR_Q_FULL = 0, BAR_K_FULL, BAR_K_EMPTY, BAR_V_FULL, BAR_V_EMPTY, BAR_S_FULL, BAR_P_FULL, BAR_PV_DONE, N_BARS };
+template <int D>
+struct Cfg {
+    static constexpr int DH = D / 64;                       // 64-channel halves per row
+    static constexpr int Q_BYTES = 128 * D * 2;
+    static constexpr int KV_BYTES = 64 * D * 2;             // one key block of K or of V
+    static constexpr int KS = (D == 128) ? 2 : 4;           // K ring stages
+    static constexpr int VS = (D == 128) ? 2 : 4;           // V ring stages
+    static constexpr int DATA_BYTES = Q_BYTES + (KS + VS) * KV_BYTES;
+};
 
 struct __align__(16) Ctl {
-    unsigned long long bars[N_BARS];
+    unsigned long long q_full;
+    unsigned long long k_full[MAX_STAGES], k_empty[MAX_STAGES];
+    unsigned long long v_full[MAX_STAGES], v_empty[MAX_STAGES];
+    unsigned long long s_full[2], p_full[2];
+    unsigned long long pv_done, o_done;
     uint32_t tmem_base;
     int n_u;
     volatile int abort_flag;
@@ -54,22 +69,26 @@ struct __align__(16) Ctl {
 };
 
 template <int D>
-__host__ __device__ constexpr int tile_bytes() { return 128 * D * 2; }
+constexpr size_t attn_smem_bytes() { return (size_t)Cfg<D>::DATA_BYTES + sizeof(Ctl) + 1024; }
 
-template <int D>
-constexpr size_t attn_smem_bytes() { return 3 * (size_t)tile_bytes<D>() + sizeof(Ctl) + 1024; }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, 2)
 attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
             const __grid_constant__ CUtensorMap tmv, const AttnParams prm) {
-    constexpr int DH = D / 64;                 // 64-channel halves per row
+    using C = Cfg<D>;
+    constexpr int DH = C::DH, KS = C::KS, VS = C::VS;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
     uint8_t* smem = smem_raw + pad;
-    const uint32_t sQ = raw + pad, sK = sQ + tile_bytes<D>(), sV = sK + tile_bytes<D>();
-    Ctl* ctl = reinterpret_cast<Ctl*>(smem + 3 * tile_bytes<D>());
+    const uint32_t sQ = raw + pad, sK = sQ + C::Q_BYTES, sV = sK + KS * C::KV_BYTES;
+    Ctl* ctl = reinterpret_cast<Ctl*>(smem + C::DATA_BYTES);
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const int pair = blockIdx.x, h = blockIdx.y, p = blockIdx.z;
@@ -79,20 +98,26 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     const int i0 = 2 * pair;
     const bool has_q1 = (i0 + 1) < nb;
 
-    uint32_t bar[N_BARS];
-#pragma unroll
-    for (int i = 0; i < N_BARS; ++i) bar[i] = smem_u32(&ctl->bars[i]);
+    const uint32_t bQ = smem_u32(&ctl->q_full), bPV = smem_u32(&ctl->pv_done), bOD = smem_u32(&ctl->o_done);
+    const uint32_t bKF = smem_u32(&ctl->k_full[0]), bKE = smem_u32(&ctl->k_empty[0]);
+    const uint32_t bVF = smem_u32(&ctl->v_full[0]), bVE = smem_u32(&ctl->v_empty[0]);
+    const uint32_t bSF = smem_u32(&ctl->s_full[0]), bPF = smem_u32(&ctl->p_full[0]);
 
     // ---------------------------------------------------------------- setup
     if (tid == 0) {
-        mbar_init(bar[BAR_Q_FULL], 1);
-        mbar_init(bar[BAR_K_FULL], 1);
-        mbar_init(bar[BAR_K_EMPTY], 1);
-        mbar_init(bar[BAR_V_FULL], 1);
-        mbar_init(bar[BAR_V_EMPTY], 1);
-        mbar_init(bar[BAR_S_FULL], 1);
-        mbar_init(bar[BAR_P_FULL], 128);
-        mbar_init(bar[BAR_PV_DONE], 1);
+        mbar_init(bQ, 1);
+        mbar_init(bPV, 1);
+        mbar_init(bOD, 1);
+        for (int s = 0; s < MAX_STAGES; ++s) {
+            mbar_init(bKF + 8 * s, 1);
+            mbar_init(bKE + 8 * s, 1);
+            mbar_init(bVF + 8 * s, 1);
+            mbar_init(bVE + 8 * s, 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bSF + 8 * s, 1);
+            mbar_init(bPF + 8 * s, 128);
+        }
         ctl->abort_flag = 0;
         ctl->n_u = 0;
         fence_mbar_init();
@@ -151,16 +176,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const int n_u = ctl->n_u;
-    const int nt = (n_u + 1) / 2;
 
     auto fail = [&]() {
         atomicExch(prm.status, RAPID3_ERR_TIMEOUT);
         ctl->abort_flag = 1;
     };
     // bounded wait that also gives up quickly once another role has failed
-    auto wait = [&](int which, uint32_t parity) -> bool {
+    auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
         for (uint32_t it = 0; it < (1u << 22); ++it) {
-            if (mbar_try_wait(bar[which], parity)) return true;
+            if (mbar_try_wait(bar, parity)) return true;
             if ((it & 255u) == 255u && ctl->abort_flag) return false;
         }
         fail();
@@ -170,68 +194,92 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     if (warp == 4) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
-            mbar_arrive_expect_tx(bar[BAR_Q_FULL], tile_bytes<D>());
+            mbar_arrive_expect_tx(bQ, C::Q_BYTES);
 #pragma unroll
             for (int c = 0; c < 2; ++c)
 #pragma unroll
                 for (int dh = 0; dh < DH; ++dh)
-                    tma_load_4d(sQ + dh * HALF_BYTES + c * BLK_BYTES, &tmq, bar[BAR_Q_FULL], dh * 64, (i0 + c) * 64, h, b);
-            int issued = 0;
-            for (int t = 0; t < nt; ++t) {
-                const int nblk = (2 * t + 1 < n_u) ? 2 : 1;
-                const int j0 = ctl->u_blk[2 * t], j1 = nblk == 2 ? ctl->u_blk[2 * t + 1] : 0;
-                if (!wait(BAR_K_EMPTY, (t & 1) ^ 1)) break;
-                mbar_arrive_expect_tx(bar[BAR_K_FULL], nblk * 64 * D * 2);
-                for (int c = 0; c < nblk; ++c)
+                    tma_load_4d(sQ + dh * QHALF_BYTES + c * BLK_BYTES, &tmq, bQ, dh * 64, (i0 + c) * 64, h, b);
+            int k_issued = 0, v_issued = 0;
+            auto load_k = [&](int j) -> bool {
+                const int s = j % KS;
+                if (!wait(bKE + 8 * s, ((j / KS) & 1) ^ 1)) return false;
+                mbar_arrive_expect_tx(bKF + 8 * s, C::KV_BYTES);
+                const int blk = ctl->u_blk[j];
 #pragma unroll
-                    for (int dh = 0; dh < DH; ++dh)
-                        tma_load_4d(sK + dh * HALF_BYTES + c * BLK_BYTES, &tmk, bar[BAR_K_FULL], dh * 64,
-                                    (c ? j1 : j0) * 64, h, b);
-                if (!wait(BAR_V_EMPTY, (t & 1) ^ 1)) { issued = 2 * t + 1; break; }
-                mbar_arrive_expect_tx(bar[BAR_V_FULL], nblk * 64 * D * 2);
-                for (int c = 0; c < nblk; ++c)
+                for (int dh = 0; dh < DH; ++dh)
+                    tma_load_4d(sK + s * C::KV_BYTES + dh * BLK_BYTES, &tmk, bKF + 8 * s, dh * 64, blk * 64, h, b);
+                k_issued = j + 1;
+                return true;
+            };
+            auto load_v = [&](int j) -> bool {
+                const int s = j % VS;
+                if (!wait(bVE + 8 * s, ((j / VS) & 1) ^ 1)) return false;
+                mbar_arrive_expect_tx(bVF + 8 * s, C::KV_BYTES);
+                const int blk = ctl->u_blk[j];
 #pragma unroll
-                    for (int dh = 0; dh < DH; ++dh)
-                        tma_load_4d(sV + dh * HALF_BYTES + c * BLK_BYTES, &tmv, bar[BAR_V_FULL], dh * 64,
-                                    (c ? j1 : j0) * 64, h, b);
-                issued = 2 * t + 2;
+                for (int dh = 0; dh < DH; ++dh)
+                    tma_load_4d(sV + s * C::KV_BYTES + dh * BLK_BYTES, &tmv, bVF + 8 * s, dh * 64, blk * 64, h, b);
+                v_issued = j + 1;
+                return true;
+            };
+            // K runs one block ahead of V, the order in which the MMA warp consumes them
+            bool ok = n_u > 0 ? load_k(0) : true;
+            for (int j = 0; ok && j < n_u; ++j) {
+                if (j + 1 < n_u && !(ok = load_k(j + 1))) break;
+                ok = load_v(j);
             }
             if (ctl->abort_flag) {
                 // drain: do not leave the CTA while bulk copies may still land in its shared memory
-                mbar_wait(bar[BAR_Q_FULL], 0, 1u << 20);
-                if (issued >= 1) mbar_wait(bar[BAR_K_FULL], ((issued - 1) / 2) & 1, 1u << 20);
-                if (issued >= 2) mbar_wait(bar[BAR_V_FULL], ((issued - 2) / 2) & 1, 1u << 20);
+                mbar_wait(bQ, 0, 1u << 20);
+                for (int j = max(0, k_issued - KS); j < k_issued; ++j)
+                    mbar_wait(bKF + 8 * (j % KS), (j / KS) & 1, 1u << 20);
+                for (int j = max(0, v_issued - VS); j < v_issued; ++j)
+                    mbar_wait(bVF + 8 * (j % VS), (j / VS) & 1, 1u << 20);
             }
         }
         __syncwarp();
     } else if (warp == 5) {
         // ------------------------------------------------------------ UMMA issue
         if (lane == 0) {
-            const uint32_t tS = tmem_base + S_COL, tO = tmem_base + O_COL;
+            const uint32_t tO = tmem_base + O_COL;
+            constexpr uint32_t idesc_qk = idesc_bf16(128, 64, 0, 0);
             constexpr uint32_t idesc_pv = idesc_bf16(128, D, 0, 1);
-            bool ok = wait(BAR_Q_FULL, 0);
-            for (int t = 0; ok && t < nt; ++t) {
-                const int nkeys = (2 * t + 1 < n_u) ? 128 : 64;
-                const uint32_t idesc_qk = idesc_bf16(128, nkeys, 0, 0);
-                if (!(ok = wait(BAR_K_FULL, t & 1))) break;
-                if (t > 0 && !(ok = wait(BAR_PV_DONE, (t - 1) & 1))) break;
+            auto issue_qk = [&](int j) -> bool {
+                const int s = j % KS;
+                if (!wait(bKF + 8 * s, (j / KS) & 1)) return false;
                 tc_fence_after();
+                const uint32_t tS = tmem_base + S_COL + 64 * (j & 1);
+                const uint32_t kb = sK + s * C::KV_BYTES;
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks / 4) * HALF_BYTES + (ks % 4) * 32;
-                    mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), idesc_qk,
-                           ks > 0);
-                }
-                tc_commit(bar[BAR_K_EMPTY]);
-                tc_commit(bar[BAR_S_FULL]);
-                if (!(ok = wait(BAR_P_FULL, t & 1))) break;
-                if (!(ok = wait(BAR_V_FULL, t & 1))) break;
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ss(tS, smem_desc_sw128(sQ + (ks / 4) * QHALF_BYTES + (ks % 4) * 32, 16, 1024),
+                           smem_desc_sw128(kb + (ks / 4) * BLK_BYTES + (ks % 4) * 32, 16, 1024), idesc_qk, ks > 0);
+                tc_commit(bKE + 8 * s);
+                tc_commit(bSF + 8 * (j & 1));
+                return true;
+            };
+            bool ok = wait(bQ, 0);
+            if (ok && n_u > 0) ok = issue_qk(0);
+            for (int j = 0; ok && j < n_u; ++j) {
+                // S(j+1) reuses the buffer of S(j-1) / P(j-1); the MMAs of this thread execute in
+                // issue order, so it is written only after P(j-1) V(j-1) has read it
+                if (j + 1 < n_u && !(ok = issue_qk(j + 1))) break;
+                if (!(ok = wait(bPF + 8 * (j & 1), (j >> 1) & 1))) break;
+                const int s = j % VS;
+                if (!(ok = wait(bVF + 8 * s, (j / VS) & 1))) break;
                 tc_fence_after();
-                for (int ks = 0; ks < nkeys / 16; ++ks)
-                    mma_ts(tO, tS + ks * 8, smem_desc_sw128(sV + ks * 2048, HALF_BYTES, 1024), idesc_pv,
-                           (t > 0 || ks > 0) ? 1u : 0u);
-                tc_commit(bar[BAR_V_EMPTY]);
-                tc_commit(bar[BAR_PV_DONE]);
+                const uint32_t tP = tmem_base + S_COL + 64 * (j & 1);
+                const uint32_t vb = sV + s * C::KV_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    mma_ts(tO, tP + ks * 8, smem_desc_sw128(vb + ks * 2048, BLK_BYTES, 1024), idesc_pv,
+                           (j > 0 || ks > 0) ? 1u : 0u);
+                tc_commit(bVE + 8 * s);
+                // pv_done advances one phase per key block (the rescale path waits on the previous
+                // block's phase); the epilogue may lag several phases, so it gets its own barrier
+                tc_commit(bPV);
+                if (j == n_u - 1) tc_commit(bOD);
             }
         }
         __syncwarp();
@@ -240,116 +288,119 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         const int a = warp >> 1;                       // which query block of the pair
         const int row = warp * 32 + lane;              // row of the 128-row tile == TMEM lane
         const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
-        const uint32_t tS = lane_addr + S_COL, tO = lane_addr + O_COL;
+        const uint32_t tO = lane_addr + O_COL;
         const float c2 = prm.scale_log2;
         const int tail_valid = N - (nb - 1) * 64;      // valid tokens of the last block (1..64)
-        float m_run = -INFINITY, l_run = 0.f;
+        float m_run = -INFINITY;
+        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
         bool ok = true;
-        uint32_t r[32];
-        for (int t = 0; t < nt; ++t) {
-            const int nhalf = (2 * t + 1 < n_u) ? 2 : 1;
-            bool act[2];
-            int valid[2];
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                const bool have = c < nhalf;
-                const int j = have ? ctl->u_blk[2 * t + c] : 0;
-                act[c] = have && ((ctl->u_flag[2 * t + c] >> a) & 1);
-                valid[c] = (j == nb - 1) ? tail_valid : 64;
-            }
-            if (!(ok = wait(BAR_S_FULL, t & 1))) break;
+        uint32_t r0[32], r1[32];
+        for (int j = 0; j < n_u; ++j) {
+            const int blk = ctl->u_blk[j];
+            const bool act = (ctl->u_flag[j] >> a) & 1;
+            const int valid = (blk == nb - 1) ? tail_valid : 64;
+            const uint32_t tS = lane_addr + S_COL + 64 * (j & 1);
+            if (!(ok = wait(bSF + 8 * (j & 1), (j >> 1) & 1))) break;
             tc_fence_after();
-            // pass 1: row maximum over the active, valid columns
-            float mx = -INFINITY;
+            if (act) {
+                tmem_ld32(tS, r0);
+                tmem_ld32(tS + 32, r1);
+                tc_wait_ld();
+                if (valid != 64) {
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                if (!act[c]) continue;
-#pragma unroll
-                for (int qd = 0; qd < 2; ++qd) {
-                    tmem_ld32(tS + c * 64 + qd * 32, r);
-                    tc_wait_ld();
-                    if (valid[c] == 64) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (qd * 32 + e < valid[c]) mx = fmaxf(mx, __uint_as_float(r[e]));
+                    for (int e = 0; e < 32; ++e) {
+                        if (e >= valid) r0[e] = 0xff800000u;          // -inf: outside the sequence
+                        if (32 + e >= valid) r1[e] = 0xff800000u;
                     }
                 }
-            }
-            // lazy rescale: move the reference maximum only when it grew by more than 2^8
-            const float m_new = fmaxf(m_run, mx);
-            const bool grow = (m_new > m_run) && ((m_new - m_run) * c2 > RESCALE_LOG2);
-            if (t > 0 && __any_sync(0xffffffffu, grow)) {
-                const float alpha = grow ? ex2((m_run - m_new) * c2) : 1.f;
-                l_run *= alpha;
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int ch = 0; ch < D / 32; ++ch) {
-                    tmem_ld32(tO + ch * 32, r);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-                    tmem_st32(tO + ch * 32, r);
+                for (int e = 0; e < 32; e += 4) {
+                    mx0 = max3(mx0, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]));
+                    mx1 = max3(mx1, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]));
+                    mx2 = max3(mx2, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]));
+                    mx3 = max3(mx3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]));
                 }
-            }
-            if (grow) m_run = m_new;
-            const float ms = m_run * c2;
-            // pass 2: P = exp2(S * c2 - ms), row sum, bf16 P over the consumed S columns
+                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                // lazy rescale: move the reference maximum only when it grew by more than 2^8
+                const float m_new = fmaxf(m_run, mx);
+                const bool grow = (m_new - m_run) * c2 > RESCALE_LOG2;    // true from -inf
+                const bool fix_o = grow && m_run != -INFINITY;            // O holds something to rescale
+                if (__any_sync(0xffffffffu, fix_o)) {
+                    // O must be at rest: wait for P(j-1) V(j-1)
+                    if (!(ok = wait(bPV, (j - 1) & 1))) break;
+                    tc_fence_after();
+                    const float alpha = fix_o ? ex2((m_run - m_new) * c2) : 1.f;
+                    l0 *= alpha; l1 *= alpha; l2 *= alpha; l3 *= alpha;
+                    uint32_t o[32];
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                if (c >= nhalf) continue;
-#pragma unroll
-                for (int qd = 0; qd < 2; ++qd) {
-                    uint32_t pk[16];
-                    if (act[c]) {
-                        tmem_ld32(tS + c * 64 + qd * 32, r);
+                    for (int ch = 0; ch < D / 32; ++ch) {
+                        tmem_ld32(tO + ch * 32, o);
                         tc_wait_ld();
-                        float pv[32];
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            float x = ex2(fmaf(__uint_as_float(r[e]), c2, -ms));
-                            if (valid[c] != 64 && qd * 32 + e >= valid[c]) x = 0.f;
-                            pv[e] = x;
-                            l_run += x;
-                        }
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) pk[e] = pack_bf16(pv[2 * e], pv[2 * e + 1]);
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) pk[e] = 0u;
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tmem_st32(tO + ch * 32, o);
                     }
-                    tmem_st16(tS + c * 32 + qd * 16, pk);
                 }
+                if (grow) m_run = m_new;
+                const float ms = m_run * c2;
+                uint32_t pk[32];
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float x0 = ex2(fmaf(__uint_as_float(r0[e]), c2, -ms));
+                    const float x1 = ex2(fmaf(__uint_as_float(r0[e + 1]), c2, -ms));
+                    const float x2 = ex2(fmaf(__uint_as_float(r0[e + 2]), c2, -ms));
+                    const float x3 = ex2(fmaf(__uint_as_float(r0[e + 3]), c2, -ms));
+                    l0 += x0; l1 += x1; l2 += x2; l3 += x3;
+                    pk[e / 2] = pack_bf16(x0, x1);
+                    pk[e / 2 + 1] = pack_bf16(x2, x3);
+                }
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    const float x0 = ex2(fmaf(__uint_as_float(r1[e]), c2, -ms));
+                    const float x1 = ex2(fmaf(__uint_as_float(r1[e + 1]), c2, -ms));
+                    const float x2 = ex2(fmaf(__uint_as_float(r1[e + 2]), c2, -ms));
+                    const float x3 = ex2(fmaf(__uint_as_float(r1[e + 3]), c2, -ms));
+                    l0 += x0; l1 += x1; l2 += x2; l3 += x3;
+                    pk[16 + e / 2] = pack_bf16(x0, x1);
+                    pk[16 + e / 2 + 1] = pack_bf16(x2, x3);
+                }
+                tmem_st32(tS, pk);
+            } else {
+                uint32_t z[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) z[e] = 0u;
+                tmem_st32(tS, z);
             }
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(bar[BAR_P_FULL]);
+            mbar_arrive(bPF + 8 * (j & 1));
         }
         // epilogue: O / l -> bf16 -> global
         const int n_glob = i0 * 64 + row;
         uint16_t* orow = prm.out + (long long)b * g.stride_b + (long long)h * g.stride_h + (long long)n_glob * g.stride_n;
-        if (ok && nt > 0) ok = wait(BAR_PV_DONE, (nt - 1) & 1);
+        if (ok && n_u > 0) ok = wait(bOD, 0);
         if (ok) {
             tc_fence_after();
+            const float l_run = (l0 + l1) + (l2 + l3);
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
 #pragma unroll
             for (int ch = 0; ch < D / 32; ++ch) {
-                if (nt > 0) {
-                    tmem_ld32(tO + ch * 32, r);
+                if (n_u > 0) {
+                    tmem_ld32(tO + ch * 32, r0);
                     tc_wait_ld();
                 } else {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) r[e] = 0u;
+                    for (int e = 0; e < 32; ++e) r0[e] = 0u;
                 }
                 if (n_glob < N) {
 #pragma unroll
                     for (int v4 = 0; v4 < 4; ++v4) {
                         uint4 o;
-                        o.x = pack_bf16(__uint_as_float(r[v4 * 8 + 0]) * inv, __uint_as_float(r[v4 * 8 + 1]) * inv);
-                        o.y = pack_bf16(__uint_as_float(r[v4 * 8 + 2]) * inv, __uint_as_float(r[v4 * 8 + 3]) * inv);
-                        o.z = pack_bf16(__uint_as_float(r[v4 * 8 + 4]) * inv, __uint_as_float(r[v4 * 8 + 5]) * inv);
-                        o.w = pack_bf16(__uint_as_float(r[v4 * 8 + 6]) * inv, __uint_as_float(r[v4 * 8 + 7]) * inv);
+                        o.x = pack_bf16(__uint_as_float(r0[v4 * 8 + 0]) * inv, __uint_as_float(r0[v4 * 8 + 1]) * inv);
+                        o.y = pack_bf16(__uint_as_float(r0[v4 * 8 + 2]) * inv, __uint_as_float(r0[v4 * 8 + 3]) * inv);
+                        o.z = pack_bf16(__uint_as_float(r0[v4 * 8 + 4]) * inv, __uint_as_float(r0[v4 * 8 + 5]) * inv);
+                        o.w = pack_bf16(__uint_as_float(r0[v4 * 8 + 6]) * inv, __uint_as_float(r0[v4 * 8 + 7]) * inv);
                         *reinterpret_cast<uint4*>(orow + ch * 32 + v4 * 8) = o;
                     }
                 }
@@ -363,8 +414,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     if (warp == 5) {
         if (ctl->abort_flag && lane == 0) {
             // make sure no UMMA is still in flight before the TMEM columns are released
-            tc_commit(bar[BAR_Q_FULL]);
-            mbar_wait(bar[BAR_Q_FULL], 1, 1u << 20);
+            tc_commit(bQ);
+            mbar_wait(bQ, 1, 1u << 20);
         }
         __syncwarp();
         tc_fence_after();
