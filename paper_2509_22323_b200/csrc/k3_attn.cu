@@ -241,36 +241,42 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         __syncwarp();
     } else if (warp == 5) {
         // ------------------------------------------------------------ UMMA issue
-        if (lane == 0) {
-            const uint32_t tO = tmem_base + O_COL;
-            constexpr uint32_t idesc_qk = idesc_bf16(128, 64, 0, 0);
-            constexpr uint32_t idesc_pv = idesc_bf16(128, D, 0, 1);
-            auto issue_qk = [&](int j) -> bool {
-                const int s = j % KS;
-                if (!wait(bKF + 8 * s, (j / KS) & 1)) return false;
-                tc_fence_after();
-                const uint32_t tS = tmem_base + S_COL + 64 * (j & 1);
-                const uint32_t kb = sK + s * C::KV_BYTES;
+        // The whole warp runs the loop converged (addresses and descriptors stay warp-uniform);
+        // one elected lane issues the tcgen05 instructions.
+        const bool leader = elect_one();
+        const uint32_t tO = tmem_base + O_COL;
+        constexpr uint32_t idesc_qk = idesc_bf16(128, 64, 0, 0);
+        constexpr uint32_t idesc_pv = idesc_bf16(128, D, 0, 1);
+        auto issue_qk = [&](int j) -> bool {
+            const int s = j % KS;
+            if (!__all_sync(0xffffffffu, wait(bKF + 8 * s, (j / KS) & 1))) return false;
+            tc_fence_after();
+            const uint32_t tS = tmem_base + S_COL + 64 * (j & 1);
+            const uint32_t kb = sK + s * C::KV_BYTES;
+            if (leader) {
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks)
                     mma_ss(tS, smem_desc_sw128(sQ + (ks / 4) * QHALF_BYTES + (ks % 4) * 32, 16, 1024),
                            smem_desc_sw128(kb + (ks / 4) * BLK_BYTES + (ks % 4) * 32, 16, 1024), idesc_qk, ks > 0);
                 tc_commit(bKE + 8 * s);
                 tc_commit(bSF + 8 * (j & 1));
-                return true;
-            };
-            bool ok = wait(bQ, 0);
-            if (ok && n_u > 0) ok = issue_qk(0);
-            for (int j = 0; ok && j < n_u; ++j) {
-                // S(j+1) reuses the buffer of S(j-1) / P(j-1); the MMAs of this thread execute in
-                // issue order, so it is written only after P(j-1) V(j-1) has read it
-                if (j + 1 < n_u && !(ok = issue_qk(j + 1))) break;
-                if (!(ok = wait(bPF + 8 * (j & 1), (j >> 1) & 1))) break;
-                const int s = j % VS;
-                if (!(ok = wait(bVF + 8 * s, (j / VS) & 1))) break;
-                tc_fence_after();
-                const uint32_t tP = tmem_base + S_COL + 64 * (j & 1);
-                const uint32_t vb = sV + s * C::KV_BYTES;
+            }
+            __syncwarp();
+            return true;
+        };
+        bool ok = __all_sync(0xffffffffu, wait(bQ, 0));
+        if (ok && n_u > 0) ok = issue_qk(0);
+        for (int j = 0; ok && j < n_u; ++j) {
+            // S(j+1) reuses the buffer of S(j-1) / P(j-1); the MMAs of the issuing thread execute in
+            // issue order, so it is written only after P(j-1) V(j-1) has read it
+            if (j + 1 < n_u && !(ok = issue_qk(j + 1))) break;
+            if (!(ok = __all_sync(0xffffffffu, wait(bPF + 8 * (j & 1), (j >> 1) & 1)))) break;
+            const int s = j % VS;
+            if (!(ok = __all_sync(0xffffffffu, wait(bVF + 8 * s, (j / VS) & 1)))) break;
+            tc_fence_after();
+            const uint32_t tP = tmem_base + S_COL + 64 * (j & 1);
+            const uint32_t vb = sV + s * C::KV_BYTES;
+            if (leader) {
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
                     mma_ts(tO, tP + ks * 8, smem_desc_sw128(vb + ks * 2048, BLK_BYTES, 1024), idesc_pv,
@@ -281,8 +287,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                 tc_commit(bPV);
                 if (j == n_u - 1) tc_commit(bOD);
             }
+            __syncwarp();
         }
-        __syncwarp();
     } else {
         // ------------------------------------------------------------ softmax / correction / epilogue
         const int a = warp >> 1;                       // which query block of the pair
