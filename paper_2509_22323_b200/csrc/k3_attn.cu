@@ -1,21 +1,25 @@
 // K3: masked flash-style joint attention over the kept key tiles (sm_100a).
 //
-// One CTA per (image, head, pair of adjacent 64-token query blocks) = a 128-row Q tile, the
-// native UMMA M.  The two query blocks' ascending kept lists are merged into one union list and
-// the CTA walks it one 64-token key block at a time.  A 64x64 sub-tile whose key block is not
-// in that query block's own list gets P = 0, so each query block attends exactly its own kept
-// set.
+// One CTA per (image, head, four adjacent 64-token query blocks) = two 128-row Q tiles (the
+// native UMMA M), one CTA per SM.  The four query blocks' ascending kept lists are merged into
+// one union list; the producer streams each key block of the union once through shared memory
+// and both tiles use it, which nearly halves the L2 -> SM traffic per MMA and leaves room for
+// deep K / V rings.  A tile issues no MMA for a key block that neither of its query blocks
+// kept; inside a tile a 64x64 sub-tile whose key block is not in that query block's own list
+// gets P = 0, so each query block attends exactly its own kept set.
 //
-// Pipeline inside a CTA (192 threads):
-//   warp 4     producer: TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of Q once, then the
-//              gathered K and V blocks into two rings of shared-memory stages
-//   warp 5     TMEM allocation and UMMA issue.  S is double buffered in TMEM (2 x 64 fp32
-//              columns): S(j+1) = Q K(j+1)^T is issued before O += P(j) V(j), so the tensor pipe
-//              works on the next scores while the softmax warps are busy with the current ones
-//   warps 0-3  softmax: thread = one query row; S(j) from TMEM in one pass (64 registers), fp32
-//              online softmax with lazy rescale of O, P(j) written back over S(j) as bf16,
-//              final O / l store
-// Two CTAs are resident per SM (2 x 256 TMEM columns, ~100 KB shared memory each).
+// Roles (352 threads):
+//   warp 8      producer: TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of Q once, then
+//               the gathered K and V blocks into two rings of shared-memory stages
+//   warps 9,10  UMMA issue, one warp per tile (warp 9 also owns the TMEM allocation).  S of a
+//               tile is double buffered in TMEM (2 x 64 fp32 columns): S(n+1) = Q K^T is issued
+//               before O += P(n) V, so the tensor pipe works on the next scores while the
+//               softmax warps are busy with the current ones.  Both warps walk the same union
+//               list one block ahead in K than in V; a stage is released when both have passed it
+//   warps 0-7   softmax, four warps per tile: thread = one query row; S(n) from TMEM in one pass
+//               (64 registers), fp32 online softmax with lazy rescale of O, P(n) written back
+//               over S(n) as bf16, final O / l store
+// TMEM: tile t owns columns [256 t, 256 t + 256): S(n) at 64 (n & 1), O at 128.
 // Every mbarrier wait is bounded; a wait that runs out records RAPID3_ERR_TIMEOUT in the status
 // word and the CTA drains its copies, releases its TMEM and exits normally.
 #include "common.cuh"
@@ -25,14 +29,15 @@ using namespace ptx;
 
 namespace {
 
-constexpr int NTHREADS = 192;
-constexpr int TMEM_COLS = 256;
-constexpr int S_COL = 0;            // S(j) at columns [64 * (j & 1), +64); P(j) over its first 32
+constexpr int NTHREADS = 352;
+constexpr int PRODUCER_WARP = 8, MMA_WARP0 = 9;
+constexpr int TMEM_COLS = 512;
+constexpr int TILE_COLS = 256;      // TMEM columns of one Q tile
 constexpr int O_COL = 128;
 constexpr int BLK_BYTES = 8192;     // 64 rows x 128 bytes: one 64-channel half of a 64-token block
-constexpr int QHALF_BYTES = 16384;  // one 64-channel half of the 128-row Q tile
+constexpr int QHALF_BYTES = 16384;  // one 64-channel half of a 128-row Q tile
 constexpr float RESCALE_LOG2 = 8.0f;
-constexpr int MAX_STAGES = 4;
+constexpr int MAX_STAGES = 8;
 
 struct AttnParams {
     TensorGeom g;
@@ -47,25 +52,25 @@ struct AttnParams {
 template <int D>
 struct Cfg {
     static constexpr int DH = D / 64;                       // 64-channel halves per row
-    static constexpr int Q_BYTES = 128 * D * 2;
+    static constexpr int QTILE_BYTES = 128 * D * 2;         // one 128-row Q tile
     static constexpr int KV_BYTES = 64 * D * 2;             // one key block of K or of V
-    static constexpr int KS = (D == 128) ? 2 : 4;           // K ring stages
-    static constexpr int VS = (D == 128) ? 2 : 4;           // V ring stages
-    static constexpr int DATA_BYTES = Q_BYTES + (KS + VS) * KV_BYTES;
+    static constexpr int KS = (D == 128) ? 4 : 8;           // K ring stages
+    static constexpr int VS = (D == 128) ? 4 : 8;           // V ring stages
+    static constexpr int DATA_BYTES = 2 * QTILE_BYTES + (KS + VS) * KV_BYTES;
 };
 
 struct __align__(16) Ctl {
     unsigned long long q_full;
     unsigned long long k_full[MAX_STAGES], k_empty[MAX_STAGES];
     unsigned long long v_full[MAX_STAGES], v_empty[MAX_STAGES];
-    unsigned long long s_full[2], p_full[2];
-    unsigned long long pv_done, o_done;
+    unsigned long long s_full[2][2], p_full[2][2];
+    unsigned long long pv_done[2], o_done[2], drain[2];
     uint32_t tmem_base;
     int n_u;
     volatile int abort_flag;
-    uint32_t bm[2][32];
+    uint32_t bm[4][32];
     int16_t u_blk[RAPID3_MAX_NB];
-    uint8_t u_flag[RAPID3_MAX_NB];
+    uint8_t u_flag[RAPID3_MAX_NB];      // bit a: query block a of the quad keeps this key block
 };
 
 template <int D>
@@ -78,7 +83,7 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 
 template <int D>
-__global__ void __launch_bounds__(NTHREADS, 2)
+__global__ void __launch_bounds__(NTHREADS, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
             const __grid_constant__ CUtensorMap tmv, const AttnParams prm) {
     using C = Cfg<D>;
@@ -87,36 +92,42 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
     uint8_t* smem = smem_raw + pad;
-    const uint32_t sQ = raw + pad, sK = sQ + C::Q_BYTES, sV = sK + KS * C::KV_BYTES;
+    const uint32_t sQ = raw + pad, sK = sQ + 2 * C::QTILE_BYTES, sV = sK + KS * C::KV_BYTES;
     Ctl* ctl = reinterpret_cast<Ctl*>(smem + C::DATA_BYTES);
 
-    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int pair = blockIdx.x, h = blockIdx.y, p = blockIdx.z;
+    const int tid = threadIdx.x, lane = tid % 32;
+    // the shuffle makes the warp index provably warp-uniform, so role branches and the address
+    // arithmetic inside them can live in uniform registers
+    const int warp = __shfl_sync(0xffffffffu, tid / 32, 0);
+    const int quad = blockIdx.x, h = blockIdx.y, p = blockIdx.z;
     const TensorGeom& g = prm.g;
     const int nb = g.nb, N = g.N;
     const int b = prm.imgs.batch[p], slot = prm.imgs.slot[p];
-    const int i0 = 2 * pair;
-    const bool has_q1 = (i0 + 1) < nb;
+    const int i0 = 4 * quad;
 
-    const uint32_t bQ = smem_u32(&ctl->q_full), bPV = smem_u32(&ctl->pv_done), bOD = smem_u32(&ctl->o_done);
+    const uint32_t bQ = smem_u32(&ctl->q_full);
     const uint32_t bKF = smem_u32(&ctl->k_full[0]), bKE = smem_u32(&ctl->k_empty[0]);
     const uint32_t bVF = smem_u32(&ctl->v_full[0]), bVE = smem_u32(&ctl->v_empty[0]);
-    const uint32_t bSF = smem_u32(&ctl->s_full[0]), bPF = smem_u32(&ctl->p_full[0]);
+    const uint32_t bSF = smem_u32(&ctl->s_full[0][0]), bPF = smem_u32(&ctl->p_full[0][0]);   // [tile][buf]: + 16 t + 8 buf
+    const uint32_t bPV = smem_u32(&ctl->pv_done[0]), bOD = smem_u32(&ctl->o_done[0]);        // [tile]: + 8 t
 
     // ---------------------------------------------------------------- setup
     if (tid == 0) {
         mbar_init(bQ, 1);
-        mbar_init(bPV, 1);
-        mbar_init(bOD, 1);
         for (int s = 0; s < MAX_STAGES; ++s) {
             mbar_init(bKF + 8 * s, 1);
-            mbar_init(bKE + 8 * s, 1);
+            mbar_init(bKE + 8 * s, 2);      // both tiles pass a stage before it is refilled
             mbar_init(bVF + 8 * s, 1);
-            mbar_init(bVE + 8 * s, 1);
+            mbar_init(bVE + 8 * s, 2);
         }
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < 4; ++s) {
             mbar_init(bSF + 8 * s, 1);
             mbar_init(bPF + 8 * s, 128);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bPV + 8 * t, 1);
+            mbar_init(bOD + 8 * t, 1);
+            mbar_init(smem_u32(&ctl->drain[t]), 1);
         }
         ctl->abort_flag = 0;
         ctl->n_u = 0;
@@ -125,17 +136,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         prefetch_tmap(&tmk);
         prefetch_tmap(&tmv);
     }
-    if (tid < 64) ctl->bm[tid / 32][tid % 32] = 0;
-    if (warp == 5) {
+    if (tid < 128) ctl->bm[tid / 32][tid % 32] = 0;
+    if (warp == MMA_WARP0) {
         tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS);
         tmem_relinquish();
         tc_fence_before();
     }
     __syncthreads();
 
-    // ---------------------------------------------------------------- union of the two kept lists
+    // ---------------------------------------------------------------- union of the four kept lists
     if (slot >= 0 && prm.kept_idx != nullptr) {
-        for (int a = 0; a < (has_q1 ? 2 : 1); ++a) {
+        for (int a = 0; a < 4 && i0 + a < nb; ++a) {
             const long long row = ((long long)slot * g.H + h) * nb + i0 + a;
             const int cnt = min(max(prm.kept_cnt[row], 0), nb);
             const int32_t* lst = prm.kept_idx + row * nb;
@@ -148,13 +159,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     } else if (tid < 32) {
         const int n = min(max(nb - tid * 32, 0), 32);
         const uint32_t val = n == 32 ? 0xffffffffu : ((1u << n) - 1u);
-        ctl->bm[0][tid] = val;
-        ctl->bm[1][tid] = has_q1 ? val : 0u;
+        for (int a = 0; a < 4; ++a) ctl->bm[a][tid] = (i0 + a < nb) ? val : 0u;
     }
     __syncthreads();
     if (warp == 0) {
-        const uint32_t m0 = ctl->bm[0][lane], m1 = ctl->bm[1][lane];
-        uint32_t u = m0 | m1;
+        const uint32_t m0 = ctl->bm[0][lane], m1 = ctl->bm[1][lane], m2 = ctl->bm[2][lane], m3 = ctl->bm[3][lane];
+        uint32_t u = m0 | m1 | m2 | m3;
         const int c = __popc(u);
         int incl = c;
 #pragma unroll
@@ -167,7 +177,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             const int bit = __ffs(u) - 1;
             u &= u - 1;
             ctl->u_blk[pos] = (int16_t)(lane * 32 + bit);
-            ctl->u_flag[pos] = (uint8_t)(((m0 >> bit) & 1u) | (((m1 >> bit) & 1u) << 1));
+            ctl->u_flag[pos] = (uint8_t)(((m0 >> bit) & 1u) | (((m1 >> bit) & 1u) << 1) | (((m2 >> bit) & 1u) << 2) |
+                                         (((m3 >> bit) & 1u) << 3));
             ++pos;
         }
         if (lane == 31) ctl->n_u = incl;
@@ -190,16 +201,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         fail();
         return false;
     };
+    // the same for a converged warp, with a warp-uniform result
+    auto wait_warp = [&](uint32_t bar, uint32_t parity) -> bool {
+        return __all_sync(0xffffffffu, wait(bar, parity));
+    };
 
-    if (warp == 4) {
+    if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
-            mbar_arrive_expect_tx(bQ, C::Q_BYTES);
+            mbar_arrive_expect_tx(bQ, 2 * C::QTILE_BYTES);
 #pragma unroll
-            for (int c = 0; c < 2; ++c)
+            for (int a = 0; a < 4; ++a)
 #pragma unroll
                 for (int dh = 0; dh < DH; ++dh)
-                    tma_load_4d(sQ + dh * QHALF_BYTES + c * BLK_BYTES, &tmq, bQ, dh * 64, (i0 + c) * 64, h, b);
+                    tma_load_4d(sQ + (a >> 1) * C::QTILE_BYTES + dh * QHALF_BYTES + (a & 1) * BLK_BYTES, &tmq, bQ,
+                                dh * 64, (i0 + a) * 64, h, b);
             int k_issued = 0, v_issued = 0;
             auto load_k = [&](int j) -> bool {
                 const int s = j % KS;
@@ -223,7 +239,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                 v_issued = j + 1;
                 return true;
             };
-            // K runs one block ahead of V, the order in which the MMA warp consumes them
+            // K runs one block ahead of V, the order in which the MMA warps consume them
             bool ok = n_u > 0 ? load_k(0) : true;
             for (int j = 0; ok && j < n_u; ++j) {
                 if (j + 1 < n_u && !(ok = load_k(j + 1))) break;
@@ -239,74 +255,101 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             }
         }
         __syncwarp();
-    } else if (warp == 5) {
-        // ------------------------------------------------------------ UMMA issue
+    } else if (warp >= MMA_WARP0) {
+        // ------------------------------------------------------------ UMMA issue, one warp per tile
         // The whole warp runs the loop converged (addresses and descriptors stay warp-uniform);
-        // one elected lane issues the tcgen05 instructions.
+        // one elected lane issues the tcgen05 instructions.  Both warps pass over every block of
+        // the union list, K one block ahead of V, also over blocks their tile does not use: the
+        // stage barriers then see every phase in order and a stage is refilled only after both
+        // tiles are past it.
+        const int t = warp - MMA_WARP0;
         const bool leader = elect_one();
-        const uint32_t tO = tmem_base + O_COL;
+        const uint32_t tbase = tmem_base + t * TILE_COLS;
+        const uint32_t tO = tbase + O_COL;
+        const uint32_t qb = sQ + t * C::QTILE_BYTES;
+        const uint32_t bSFt = bSF + 16 * t, bPFt = bPF + 16 * t;
         constexpr uint32_t idesc_qk = idesc_bf16(128, 64, 0, 0);
         constexpr uint32_t idesc_pv = idesc_bf16(128, D, 0, 1);
-        auto issue_qk = [&](int j) -> bool {
+        int n_qk = 0, n_pv = 0;                        // blocks of this tile issued so far
+        auto k_step = [&](int j) -> bool {
             const int s = j % KS;
-            if (!__all_sync(0xffffffffu, wait(bKF + 8 * s, (j / KS) & 1))) return false;
-            tc_fence_after();
-            const uint32_t tS = tmem_base + S_COL + 64 * (j & 1);
-            const uint32_t kb = sK + s * C::KV_BYTES;
-            if (leader) {
+            const bool use = (ctl->u_flag[j] >> (2 * t)) & 3u;
+            if (!(wait_warp(bKF + 8 * s, (j / KS) & 1))) return false;
+            if (use) {
+                tc_fence_after();
+                const uint32_t tS = tbase + 64 * (n_qk & 1);
+                const uint32_t kb = sK + s * C::KV_BYTES;
+                if (leader) {
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(tS, smem_desc_sw128(sQ + (ks / 4) * QHALF_BYTES + (ks % 4) * 32, 16, 1024),
-                           smem_desc_sw128(kb + (ks / 4) * BLK_BYTES + (ks % 4) * 32, 16, 1024), idesc_qk, ks > 0);
-                tc_commit(bKE + 8 * s);
-                tc_commit(bSF + 8 * (j & 1));
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        mma_ss(tS, smem_desc_sw128(qb + (ks / 4) * QHALF_BYTES + (ks % 4) * 32, 16, 1024),
+                               smem_desc_sw128(kb + (ks / 4) * BLK_BYTES + (ks % 4) * 32, 16, 1024), idesc_qk, ks > 0);
+                    tc_commit(bKE + 8 * s);
+                    tc_commit(bSFt + 8 * (n_qk & 1));
+                }
+                ++n_qk;
+            } else if (leader) {
+                mbar_arrive(bKE + 8 * s);
             }
             __syncwarp();
             return true;
         };
-        bool ok = __all_sync(0xffffffffu, wait(bQ, 0));
-        if (ok && n_u > 0) ok = issue_qk(0);
+        bool ok = (wait_warp(bQ, 0));
+        if (ok && n_u > 0) ok = k_step(0);
         for (int j = 0; ok && j < n_u; ++j) {
-            // S(j+1) reuses the buffer of S(j-1) / P(j-1); the MMAs of the issuing thread execute in
-            // issue order, so it is written only after P(j-1) V(j-1) has read it
-            if (j + 1 < n_u && !(ok = issue_qk(j + 1))) break;
-            if (!(ok = __all_sync(0xffffffffu, wait(bPF + 8 * (j & 1), (j >> 1) & 1)))) break;
+            // S(n+1) reuses the buffer of P(n-1); the MMAs of the issuing thread execute in issue
+            // order, so it is written only after P(n-1) V has read it
+            if (j + 1 < n_u && !(ok = k_step(j + 1))) break;
             const int s = j % VS;
-            if (!(ok = __all_sync(0xffffffffu, wait(bVF + 8 * s, (j / VS) & 1)))) break;
-            tc_fence_after();
-            const uint32_t tP = tmem_base + S_COL + 64 * (j & 1);
-            const uint32_t vb = sV + s * C::KV_BYTES;
-            if (leader) {
+            const bool use = (ctl->u_flag[j] >> (2 * t)) & 3u;
+            if (use && !(ok = (wait_warp(bPFt + 8 * (n_pv & 1), (n_pv >> 1) & 1)))) break;
+            if (!(ok = (wait_warp(bVF + 8 * s, (j / VS) & 1)))) break;
+            if (use) {
+                tc_fence_after();
+                const uint32_t tP = tbase + 64 * (n_pv & 1);
+                const uint32_t vb = sV + s * C::KV_BYTES;
+                if (leader) {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    mma_ts(tO, tP + ks * 8, smem_desc_sw128(vb + ks * 2048, BLK_BYTES, 1024), idesc_pv,
-                           (j > 0 || ks > 0) ? 1u : 0u);
-                tc_commit(bVE + 8 * s);
-                // pv_done advances one phase per key block (the rescale path waits on the previous
-                // block's phase); the epilogue may lag several phases, so it gets its own barrier
-                tc_commit(bPV);
-                if (j == n_u - 1) tc_commit(bOD);
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_ts(tO, tP + ks * 8, smem_desc_sw128(vb + ks * 2048, BLK_BYTES, 1024), idesc_pv,
+                               (n_pv > 0 || ks > 0) ? 1u : 0u);
+                    tc_commit(bVE + 8 * s);
+                    // pv_done advances one phase per block of the tile (the rescale path waits on the
+                    // previous block's phase); the epilogue may lag, so it has its own barrier
+                    tc_commit(bPV + 8 * t);
+                }
+                ++n_pv;
+            } else if (leader) {
+                mbar_arrive(bVE + 8 * s);
             }
             __syncwarp();
         }
+        if (ok && leader && n_pv > 0) tc_commit(bOD + 8 * t);
+        __syncwarp();
     } else {
         // ------------------------------------------------------------ softmax / correction / epilogue
-        const int a = warp >> 1;                       // which query block of the pair
-        const int row = warp * 32 + lane;              // row of the 128-row tile == TMEM lane
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const int t = warp >> 2, wl = warp & 3;        // tile, lane quarter of the tile
+        const int a = 2 * t + (wl >> 1);               // query block of the quad
+        const int row = wl * 32 + lane;                // row of the 128-row tile == TMEM lane
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(wl * 32) << 16) + t * TILE_COLS;
         const uint32_t tO = lane_addr + O_COL;
+        const uint32_t bSFt = bSF + 16 * t, bPFt = bPF + 16 * t, bPVt = bPV + 8 * t;
         const float c2 = prm.scale_log2;
         const int tail_valid = N - (nb - 1) * 64;      // valid tokens of the last block (1..64)
         float m_run = -INFINITY;
         float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
         bool ok = true;
         uint32_t r0[32], r1[32];
+        int n = 0;                                     // blocks of this tile so far
         for (int j = 0; j < n_u; ++j) {
+            const uint32_t f = ctl->u_flag[j];
+            if (!((f >> (2 * t)) & 3u)) continue;      // neither query block of the tile kept it
             const int blk = ctl->u_blk[j];
-            const bool act = (ctl->u_flag[j] >> a) & 1;
+            const bool act = (f >> a) & 1u;
             const int valid = (blk == nb - 1) ? tail_valid : 64;
-            const uint32_t tS = lane_addr + S_COL + 64 * (j & 1);
-            if (!(ok = wait(bSF + 8 * (j & 1), (j >> 1) & 1))) break;
+            const int buf = n & 1;
+            const uint32_t tS = lane_addr + 64 * buf;
+            if (!(ok = wait_warp(bSFt + 8 * buf, (n >> 1) & 1))) break;
             tc_fence_after();
             if (act) {
                 tmem_ld32(tS, r0);
@@ -333,8 +376,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                 const bool grow = (m_new - m_run) * c2 > RESCALE_LOG2;    // true from -inf
                 const bool fix_o = grow && m_run != -INFINITY;            // O holds something to rescale
                 if (__any_sync(0xffffffffu, fix_o)) {
-                    // O must be at rest: wait for P(j-1) V(j-1)
-                    if (!(ok = wait(bPV, (j - 1) & 1))) break;
+                    // O must be at rest: wait for P(n-1) V
+                    if (!(ok = wait_warp(bPVt, (n - 1) & 1))) break;
                     tc_fence_after();
                     const float alpha = fix_o ? ex2((m_run - m_new) * c2) : 1.f;
                     l0 *= alpha; l1 *= alpha; l2 *= alpha; l3 *= alpha;
@@ -380,19 +423,20 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             }
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(bPF + 8 * (j & 1));
+            mbar_arrive(bPFt + 8 * buf);
+            ++n;
         }
         // epilogue: O / l -> bf16 -> global
-        const int n_glob = i0 * 64 + row;
+        const int n_glob = (i0 + 2 * t) * 64 + row;
         uint16_t* orow = prm.out + (long long)b * g.stride_b + (long long)h * g.stride_h + (long long)n_glob * g.stride_n;
-        if (ok && n_u > 0) ok = wait(bOD, 0);
+        if (ok && n > 0) ok = wait_warp(bOD + 8 * t, 0);
         if (ok) {
             tc_fence_after();
             const float l_run = (l0 + l1) + (l2 + l3);
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
 #pragma unroll
             for (int ch = 0; ch < D / 32; ++ch) {
-                if (n_u > 0) {
+                if (n > 0) {
                     tmem_ld32(tO + ch * 32, r0);
                     tc_wait_ld();
                 } else {
@@ -417,13 +461,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
-        if (ctl->abort_flag && lane == 0) {
-            // make sure no UMMA is still in flight before the TMEM columns are released
-            tc_commit(bQ);
-            mbar_wait(bQ, 1, 1u << 20);
+    if (warp >= MMA_WARP0) {
+        if (ctl->abort_flag) {
+            // make sure no UMMA of this warp is still in flight before the TMEM columns are released
+            const uint32_t bT = smem_u32(&ctl->drain[warp - MMA_WARP0]);
+            if (elect_one()) {
+                tc_commit(bT);
+                mbar_wait(bT, 0, 1u << 20);
+            }
+            __syncwarp();
         }
-        __syncwarp();
+    }
+    __syncthreads();
+    if (warp == MMA_WARP0) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
@@ -458,7 +508,7 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
     prm.out = reinterpret_cast<uint16_t*>(out);
     prm.status = status;
     prm.scale_log2 = softmax_scale * 1.4426950408889634f;
-    dim3 grid((g.nb + 1) / 2, g.H, imgs.n);
+    dim3 grid((g.nb + 3) / 4, g.H, imgs.n);
     if (g.D == 128)
         attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, prm);
     else
