@@ -187,6 +187,24 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------------------- multi-rank plumbing
+def rank_step(rank: int, s: int) -> int:
+    """Step index a rank draws its inputs with: every rank gets its own batch (weak scaling)."""
+    return rank * 1000 + s
+
+
+def aggregate(dist, device, ms_total: float, flops_total: float, launches: int):
+    """Whole-job figures from per-rank ones: the slowest rank's time, the sum of the work.
+    `dist` is torch.distributed (any backend) or None for a single process."""
+    if dist is None:
+        return ms_total, flops_total, launches
+    t = torch.tensor([ms_total], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    f = torch.tensor([flops_total, float(launches)], device=device, dtype=torch.float64)
+    dist.all_reduce(f, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(f[0].item()), int(f[1].item())
+
+
 # ----------------------------------------------------------------------------- CUDA arm
 def run_ours(args, wl):
     from paper_2509_22323_b200 import binding
@@ -211,7 +229,7 @@ def run_ours(args, wl):
         steps_of = list(range(wl.steps))           # the gated trajectory: fresh Q/K/V per step
         nsets = min(wl.steps, 4)
     # each rank draws its own data (weak scaling): shift the step index by the rank
-    sets = [inputs.make_qkv(wl, rank * 1000 + s, device=dev) for s in range(nsets)]
+    sets = [inputs.make_qkv(wl, rank_step(rank, s), device=dev) for s in range(nsets)]
     out = torch.empty_like(sets[0][0])
     plan = [(sets[i % nsets],) + tuple(inputs.make_actions(wl, steps_of[i % len(steps_of)])) for i in range(len(steps_of))]
 
@@ -270,13 +288,7 @@ def run_ours(args, wl):
         time.sleep(0.2)
         sampler.stop()
     flops_total = sum(flops_step[i % len(plan)] for i in range(args.steps))
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-        f = torch.tensor([flops_total, float(launches)], device=dev, dtype=torch.float64)
-        dist.all_reduce(f, op=dist.ReduceOp.SUM)
-        flops_total, launches = float(f[0].item()), int(f[1].item())
+    ms_total, flops_total, launches = aggregate(dist, dev, ms_total, flops_total, launches)
     value = flops_total / (ms_total * 1e-3) / 1e12
 
     # ---- end to end through the host-buffer entry point (rank-local, then max over ranks)
