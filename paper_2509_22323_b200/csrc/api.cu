@@ -134,7 +134,8 @@ int get_map(rapid3_ctx* c, const void* base, const CUtensorMap** out) {
 }
 
 int attn_launch(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out, const ImgList& l,
-                const int32_t* kept_idx, const int32_t* kept_cnt, float scale, cudaStream_t st) {
+                const int32_t* kept_idx, const int32_t* kept_cnt, const uint64_t* bitmask, float scale,
+                cudaStream_t st) {
     const CUtensorMap *mq, *mk, *mv;
     int r;
     if ((r = get_map(c, q, &mq)) || (r = get_map(c, k, &mk)) || (r = get_map(c, v, &mv))) return r;
@@ -142,7 +143,7 @@ int attn_launch(rapid3_ctx* c, const void* q, const void* k, const void* v, void
     CUtensorMap tq = *mq, tk = *mk, tv = *mv;   // copies: a later get_map may recycle the slot
     {
         ProfScope ps(c, PROF_ATTN, st);
-        if (launch_attention(tq, tk, tv, out, c->g, l, kept_idx, kept_cnt, scale, c->status, st) != cudaSuccess)
+        if (launch_attention(tq, tk, tv, out, c->g, l, kept_idx, kept_cnt, bitmask, scale, c->status, st) != cudaSuccess)
             return RAPID3_ERR_CUDA;
     }
     c->launches += 1;
@@ -293,7 +294,8 @@ int rapid3_sparse_joint_attn(rapid3_ctx* c, const void* q, const void* k, const 
     if (r != RAPID3_OK) return r;
     if (!kept_idx)
         for (int p = 0; p < n_img; ++p) l.slot[p] = -1;
-    return attn_launch(c, q, k, v, out, l, kept_idx, kept_cnt, softmax_scale, static_cast<cudaStream_t>(stream));
+    return attn_launch(c, q, k, v, out, l, kept_idx, kept_cnt, nullptr, softmax_scale,
+                       static_cast<cudaStream_t>(stream));
 }
 
 int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
@@ -354,7 +356,7 @@ int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v
         c->launches += 3;
     }
     return attn_launch(c, q, k, v, out, all, sparse.n ? c->kept_idx : nullptr, sparse.n ? c->kept_cnt : nullptr,
-                       softmax_scale, st);
+                       sparse.n ? c->bitmask : nullptr, softmax_scale, st);
 }
 
 int rapid3_gated_step_host(rapid3_ctx* c, const void* q_host, const void* k_host, const void* v_host, void* out_host,

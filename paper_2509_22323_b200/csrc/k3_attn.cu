@@ -44,6 +44,9 @@ struct AttnParams {
     ImgList imgs;
     const int32_t* kept_idx;
     const int32_t* kept_cnt;
+    const uint32_t* bitmask32;     // optional: the same mask as 32-bit words, [slot][H][nb][words32]
+    int words32;
+    int n_dense;                   // leading images of the list that keep every block
     uint16_t* out;
     int* status;
     float scale_log2;
@@ -99,9 +102,32 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     // the shuffle makes the warp index provably warp-uniform, so role branches and the address
     // arithmetic inside them can live in uniform registers
     const int warp = __shfl_sync(0xffffffffu, tid / 32, 0);
-    const int quad = blockIdx.x, h = blockIdx.y, p = blockIdx.z;
     const TensorGeom& g = prm.g;
     const int nb = g.nb, N = g.N;
+    // Work order, longest first (CTAs start in block-index order as SMs free up, so this is
+    // longest-processing-time-first scheduling): every quad of the dense images and the quads of
+    // the sparse images that hold a text query block walk all nb key blocks; the other quads of the
+    // sparse images follow, image by image in the list's order (descending keep ratio).
+    int quad, h, p;
+    {
+        const int nq = (nb + 3) >> 2, ntq = min(nq, (g.n_text_blocks + 3) >> 2);
+        const int nd = prm.n_dense, ns = prm.imgs.n - nd;
+        int L = blockIdx.x;
+        const int heavy_dense = nd * g.H * nq, heavy_sparse = ns * g.H * ntq;
+        if (L < heavy_dense) {
+            p = L / (g.H * nq); L -= p * g.H * nq;
+            h = L / nq; quad = L - h * nq;
+        } else if (L < heavy_dense + heavy_sparse) {
+            L -= heavy_dense;
+            p = L / (g.H * ntq); L -= p * g.H * ntq; p += nd;
+            h = L / ntq; quad = L - h * ntq;
+        } else {
+            L -= heavy_dense + heavy_sparse;
+            const int nl = nq - ntq;
+            p = L / (g.H * nl); L -= p * g.H * nl; p += nd;
+            h = L / nl; quad = ntq + (L - h * nl);
+        }
+    }
     const int b = prm.imgs.batch[p], slot = prm.imgs.slot[p];
     const int i0 = 4 * quad;
 
@@ -144,8 +170,28 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     }
     __syncthreads();
 
+    // The Q tiles do not depend on the mask: start their loads before the union list is built.
+    if (warp == PRODUCER_WARP && lane == 0) {
+        mbar_arrive_expect_tx(bQ, 2 * C::QTILE_BYTES);
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int dh = 0; dh < DH; ++dh)
+                tma_load_4d(sQ + (a >> 1) * C::QTILE_BYTES + dh * QHALF_BYTES + (a & 1) * BLK_BYTES, &tmq, bQ,
+                            dh * 64, (i0 + a) * 64, h, b);
+    }
+
     // ---------------------------------------------------------------- union of the four kept lists
-    if (slot >= 0 && prm.kept_idx != nullptr) {
+    // bm[a] = bit set of the key blocks query block a keeps: copied from the bitmask when the
+    // caller has one, else rebuilt from the kept list; every block is kept for a dense image.
+    const int nw = (nb + 31) >> 5;
+    if (slot >= 0 && prm.bitmask32 != nullptr) {
+        if (tid < 4 * nw) {
+            const int a = tid / nw, w = tid - a * nw;
+            if (i0 + a < nb)
+                ctl->bm[a][w] = prm.bitmask32[(((long long)slot * g.H + h) * nb + i0 + a) * prm.words32 + w];
+        }
+    } else if (slot >= 0 && prm.kept_idx != nullptr) {
         for (int a = 0; a < 4 && i0 + a < nb; ++a) {
             const long long row = ((long long)slot * g.H + h) * nb + i0 + a;
             const int cnt = min(max(prm.kept_cnt[row], 0), nb);
@@ -162,26 +208,24 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         for (int a = 0; a < 4; ++a) ctl->bm[a][tid] = (i0 + a < nb) ? val : 0u;
     }
     __syncthreads();
-    if (warp == 0) {
-        const uint32_t m0 = ctl->bm[0][lane], m1 = ctl->bm[1][lane], m2 = ctl->bm[2][lane], m3 = ctl->bm[3][lane];
-        uint32_t u = m0 | m1 | m2 | m3;
-        const int c = __popc(u);
-        int incl = c;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        int pos = incl - c;
-        while (u) {
-            const int bit = __ffs(u) - 1;
-            u &= u - 1;
-            ctl->u_blk[pos] = (int16_t)(lane * 32 + bit);
+    // one thread per key block: its position in the ascending union list is the number of union
+    // bits below it
+    for (int j = tid; j < nb; j += NTHREADS) {
+        const int w = j >> 5, bit = j & 31;
+        const uint32_t m0 = ctl->bm[0][w], m1 = ctl->bm[1][w], m2 = ctl->bm[2][w], m3 = ctl->bm[3][w];
+        const uint32_t u = m0 | m1 | m2 | m3;
+        if ((u >> bit) & 1u) {
+            int pos = __popc(u & ((1u << bit) - 1u));
+            for (int x = 0; x < w; ++x) pos += __popc(ctl->bm[0][x] | ctl->bm[1][x] | ctl->bm[2][x] | ctl->bm[3][x]);
+            ctl->u_blk[pos] = (int16_t)j;
             ctl->u_flag[pos] = (uint8_t)(((m0 >> bit) & 1u) | (((m1 >> bit) & 1u) << 1) | (((m2 >> bit) & 1u) << 2) |
                                          (((m3 >> bit) & 1u) << 3));
-            ++pos;
         }
-        if (lane == 31) ctl->n_u = incl;
+    }
+    if (tid == 0) {
+        int tot = 0;
+        for (int x = 0; x < nw; ++x) tot += __popc(ctl->bm[0][x] | ctl->bm[1][x] | ctl->bm[2][x] | ctl->bm[3][x]);
+        ctl->n_u = tot;
     }
     __syncthreads();
     tc_fence_after();
@@ -209,13 +253,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
-            mbar_arrive_expect_tx(bQ, 2 * C::QTILE_BYTES);
-#pragma unroll
-            for (int a = 0; a < 4; ++a)
-#pragma unroll
-                for (int dh = 0; dh < DH; ++dh)
-                    tma_load_4d(sQ + (a >> 1) * C::QTILE_BYTES + dh * QHALF_BYTES + (a & 1) * BLK_BYTES, &tmq, bQ,
-                                dh * 64, (i0 + a) * 64, h, b);
             int k_issued = 0, v_issued = 0;
             auto load_k = [&](int j) -> bool {
                 const int s = j % KS;
@@ -495,7 +532,8 @@ cudaError_t attention_static_init() {
 
 cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv, void* out,
                              const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
-                             const int32_t* kept_cnt, float softmax_scale, int* status, cudaStream_t s) {
+                             const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* status,
+                             cudaStream_t s) {
     if (!g_attr_set) {
         cudaError_t e = attention_static_init();
         if (e != cudaSuccess) return e;
@@ -505,10 +543,15 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
     prm.imgs = imgs;
     prm.kept_idx = kept_idx;
     prm.kept_cnt = kept_cnt;
+    prm.bitmask32 = reinterpret_cast<const uint32_t*>(bitmask);
+    prm.words32 = 2 * ((g.nb + 63) / 64);
     prm.out = reinterpret_cast<uint16_t*>(out);
     prm.status = status;
     prm.scale_log2 = softmax_scale * 1.4426950408889634f;
-    dim3 grid((g.nb + 3) / 4, g.H, imgs.n);
+    int n_dense = 0;
+    while (n_dense < imgs.n && (imgs.slot[n_dense] < 0 || kept_idx == nullptr)) ++n_dense;
+    prm.n_dense = n_dense;
+    dim3 grid(((g.nb + 3) / 4) * g.H * imgs.n, 1, 1);
     if (g.D == 128)
         attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, prm);
     else
