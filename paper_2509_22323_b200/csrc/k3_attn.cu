@@ -47,7 +47,6 @@ struct AttnParams {
     const uint32_t* bitmask32;     // optional: the same mask as 32-bit words, [slot][H][nb][words32]
     int words32;
     int n_dense;                   // leading images of the list that keep every block
-    uint16_t* out;
     int* status;
     float scale_log2;
 };
@@ -88,7 +87,7 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
-            const __grid_constant__ CUtensorMap tmv, const AttnParams prm) {
+            const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo, const AttnParams prm) {
     using C = Cfg<D>;
     constexpr int DH = C::DH, KS = C::KS, VS = C::VS;
     extern __shared__ uint8_t smem_raw[];
@@ -161,6 +160,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         prefetch_tmap(&tmq);
         prefetch_tmap(&tmk);
         prefetch_tmap(&tmv);
+        prefetch_tmap(&tmo);
     }
     if (tid < 128) ctl->bm[tid / 32][tid % 32] = 0;
     if (warp == MMA_WARP0) {
@@ -463,14 +463,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             mbar_arrive(bPFt + 8 * buf);
             ++n;
         }
-        // epilogue: O / l -> bf16 -> global
-        const int n_glob = (i0 + 2 * t) * 64 + row;
-        uint16_t* orow = prm.out + (long long)b * g.stride_b + (long long)h * g.stride_h + (long long)n_glob * g.stride_n;
+        // epilogue: O / l -> bf16 -> the tile's (now unused) Q buffer in the 128-byte swizzled layout
+        // of the tensor map -> TMA stores, one per (query block, 64-channel half); rows past the
+        // end of the sequence are clipped by the store
         if (ok && n > 0) ok = wait_warp(bOD + 8 * t, 0);
         if (ok) {
             tc_fence_after();
             const float l_run = (l0 + l1) + (l2 + l3);
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            uint8_t* so = smem + t * C::QTILE_BYTES + row * 128;
 #pragma unroll
             for (int ch = 0; ch < D / 32; ++ch) {
                 if (n > 0) {
@@ -480,18 +481,29 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
 #pragma unroll
                     for (int e = 0; e < 32; ++e) r0[e] = 0u;
                 }
-                if (n_glob < N) {
 #pragma unroll
-                    for (int v4 = 0; v4 < 4; ++v4) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(r0[v4 * 8 + 0]) * inv, __uint_as_float(r0[v4 * 8 + 1]) * inv);
-                        o.y = pack_bf16(__uint_as_float(r0[v4 * 8 + 2]) * inv, __uint_as_float(r0[v4 * 8 + 3]) * inv);
-                        o.z = pack_bf16(__uint_as_float(r0[v4 * 8 + 4]) * inv, __uint_as_float(r0[v4 * 8 + 5]) * inv);
-                        o.w = pack_bf16(__uint_as_float(r0[v4 * 8 + 6]) * inv, __uint_as_float(r0[v4 * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(orow + ch * 32 + v4 * 8) = o;
-                    }
+                for (int v4 = 0; v4 < 4; ++v4) {
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(r0[v4 * 8 + 0]) * inv, __uint_as_float(r0[v4 * 8 + 1]) * inv);
+                    o.y = pack_bf16(__uint_as_float(r0[v4 * 8 + 2]) * inv, __uint_as_float(r0[v4 * 8 + 3]) * inv);
+                    o.z = pack_bf16(__uint_as_float(r0[v4 * 8 + 4]) * inv, __uint_as_float(r0[v4 * 8 + 5]) * inv);
+                    o.w = pack_bf16(__uint_as_float(r0[v4 * 8 + 6]) * inv, __uint_as_float(r0[v4 * 8 + 7]) * inv);
+                    const int chunk = (ch & 1) * 4 + v4;            // 16-byte chunk of the 128-byte half row
+                    *reinterpret_cast<uint4*>(so + (ch >> 1) * QHALF_BYTES + ((chunk ^ (row & 7)) << 4)) = o;
                 }
             }
+            fence_proxy_async_smem();
+        }
+        // the two warps of a query block meet, then one lane stores the block
+        const int qb_id = 2 * t + (wl >> 1);
+        named_barrier_sync(1 + qb_id, 64);
+        if (ok && (wl & 1) == 0 && lane == 0 && (i0 + qb_id) * 64 < N) {
+#pragma unroll
+            for (int dh = 0; dh < DH; ++dh)
+                tma_store_4d(&tmo, sQ + t * C::QTILE_BYTES + dh * QHALF_BYTES + (wl >> 1) * BLK_BYTES, dh * 64,
+                             (i0 + qb_id) * 64, h, b);
+            bulk_commit_group();
+            bulk_wait_read_all();
         }
     }
 
@@ -530,7 +542,8 @@ cudaError_t attention_static_init() {
     return cudaSuccess;
 }
 
-cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv, void* out,
+cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv,
+                             const CUtensorMap& tmo,
                              const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
                              const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* status,
                              cudaStream_t s) {
@@ -545,7 +558,6 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
     prm.kept_cnt = kept_cnt;
     prm.bitmask32 = reinterpret_cast<const uint32_t*>(bitmask);
     prm.words32 = 2 * ((g.nb + 63) / 64);
-    prm.out = reinterpret_cast<uint16_t*>(out);
     prm.status = status;
     prm.scale_log2 = softmax_scale * 1.4426950408889634f;
     int n_dense = 0;
@@ -553,8 +565,8 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
     prm.n_dense = n_dense;
     dim3 grid(((g.nb + 3) / 4) * g.H * imgs.n, 1, 1);
     if (g.D == 128)
-        attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, prm);
+        attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, tmo, prm);
     else
-        attn_kernel<64><<<grid, NTHREADS, attn_smem_bytes<64>(), s>>>(tmq, tmk, tmv, prm);
+        attn_kernel<64><<<grid, NTHREADS, attn_smem_bytes<64>(), s>>>(tmq, tmk, tmv, tmo, prm);
     return cudaGetLastError();
 }
