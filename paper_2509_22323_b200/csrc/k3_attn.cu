@@ -433,21 +433,23 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                 uint32_t pk[32];
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
-                    const float x0 = ex2(fmaf(__uint_as_float(r0[e]), c2, -ms));
-                    const float x1 = ex2(fmaf(__uint_as_float(r0[e + 1]), c2, -ms));
-                    const float x2 = ex2(fmaf(__uint_as_float(r0[e + 2]), c2, -ms));
-                    const float x3 = ex2(fmaf(__uint_as_float(r0[e + 3]), c2, -ms));
-                    l0 += x0; l1 += x1; l2 += x2; l3 += x3;
+                    float x0, x1, x2, x3;
+                    fma2(x0, x1, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]), c2, -ms);
+                    fma2(x2, x3, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]), c2, -ms);
+                    x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
+                    add2(l0, l1, x0, x1);
+                    add2(l2, l3, x2, x3);
                     pk[e / 2] = pack_bf16(x0, x1);
                     pk[e / 2 + 1] = pack_bf16(x2, x3);
                 }
 #pragma unroll
                 for (int e = 0; e < 32; e += 4) {
-                    const float x0 = ex2(fmaf(__uint_as_float(r1[e]), c2, -ms));
-                    const float x1 = ex2(fmaf(__uint_as_float(r1[e + 1]), c2, -ms));
-                    const float x2 = ex2(fmaf(__uint_as_float(r1[e + 2]), c2, -ms));
-                    const float x3 = ex2(fmaf(__uint_as_float(r1[e + 3]), c2, -ms));
-                    l0 += x0; l1 += x1; l2 += x2; l3 += x3;
+                    float x0, x1, x2, x3;
+                    fma2(x0, x1, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]), c2, -ms);
+                    fma2(x2, x3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]), c2, -ms);
+                    x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
+                    add2(l0, l1, x0, x1);
+                    add2(l2, l3, x2, x3);
                     pk[16 + e / 2] = pack_bf16(x0, x1);
                     pk[16 + e / 2 + 1] = pack_bf16(x2, x3);
                 }
