@@ -1,8 +1,12 @@
 // K2: per (image, head, query-block row) forced + top-k block selection.
-// One warp per row.  The row of fp32 scores is staged in shared memory; every free candidate
-// gets its rank by counting the candidates that beat it under (score descending, index
-// ascending); rank < k keeps it.  The bitmask is assembled with warp ballots and the ascending
-// kept list with ballot prefix counts, so the row is written in one pass.
+// One warp per row.  The row of fp32 scores is staged in shared memory as order-preserving
+// 32-bit keys.  The k-th largest free candidate is found by a radix select over the key bits
+// (32 rounds of count-and-narrow, counts by lane-local sums and one warp reduction; rows with
+// fewer than ~100 candidates rank each candidate by counting instead); a free
+// candidate is kept when its key is above that threshold, or equal to it and among the first
+// (lowest block index) of the equal ones still needed -- the order "score descending, index
+// ascending".  The bitmask is assembled with warp ballots and the ascending kept list with ballot
+// prefix counts, so the row is written in one pass.
 #include "common.cuh"
 
 namespace {
@@ -23,31 +27,66 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
     const int i = (int)(row % nb);
     const int p = (int)(row / ((long long)nb * g.H));
     const int k = imgs.k_free[p];
-    float* s = srow + warp * nb_pad;
+    uint32_t* s = reinterpret_cast<uint32_t*>(srow) + warp * nb_pad;
     const float* src = scores + row * nb;
-    for (int j = lane; j < nb; j += 32) s[j] = src[j];
-    __syncwarp();
-
     const bool text_row = i < ntb;
+    // key: unsigned integer with the same order as the float (-0 and +0 made equal)
+    for (int j = lane; j < nb_pad; j += 32) {
+        uint32_t u = 0u;
+        if (j < nb) {
+            u = __float_as_uint(src[j]);
+            if (u == 0x80000000u) u = 0u;
+            u ^= (u >> 31) ? 0xffffffffu : 0x80000000u;
+        }
+        s[j] = u;
+    }
+    __syncwarp();
+    const int n_free = max(nb - ntb - ((i >= ntb) ? 1 : 0), 0);
+    // radix select of the k-th largest key among the free candidates
+    uint32_t prefix = 0u, mask = 0u;
+    int want = k;                                       // rank still looked for inside the prefix group
+    const bool select = !text_row && k > 0 && k < n_free;
+    const bool radix = n_free > 96;                     // short rows: ranking by counting is cheaper than 32 rounds
+    if (select && radix) {
+        for (int bit = 31; bit >= 0; --bit) {
+            const uint32_t trial = prefix | (1u << bit), m2 = mask | (1u << bit);
+            int cnt = 0;
+            for (int j = lane; j < nb; j += 32) cnt += (j >= ntb) && (j != i) && ((s[j] & m2) == trial);
+            cnt = __reduce_add_sync(0xffffffffu, cnt);
+            if (cnt >= want) prefix = trial;
+            else want -= cnt;
+            mask = m2;
+        }
+    }
     int32_t* out_idx = kept_idx + row * nb;
     uint32_t* out_bits = bitmask32 + row * words32;
-    int total = 0;
+    int total = 0, eq_seen = 0;
     for (int c = 0; c < nb_pad; c += 32) {
         const int j = c + lane;
-        bool keep = false;
+        bool keep = false, eq = false;
         if (j < nb) {
             if (text_row || j < ntb || j == i) {
                 keep = true;
-            } else {
-                const float sj = s[j];
+            } else if (select && radix) {
+                keep = s[j] > prefix;
+                eq = s[j] == prefix;
+            } else if (select) {
+                // rank = number of free candidates that beat this one (key descending, index ascending)
+                const uint32_t sj = s[j];
                 int rank = 0;
                 for (int m = ntb; m < nb; ++m) {
-                    const float sm = s[m];
+                    const uint32_t sm = s[m];
                     rank += (m != i) && (sm > sj || (sm == sj && m < j));
                 }
                 keep = rank < k;
+            } else {
+                keep = k >= n_free && k > 0;            // every free candidate, or none
             }
         }
+        // equal keys: the lowest block indices first, `want` of them in all
+        const uint32_t beq = __ballot_sync(0xffffffffu, eq);
+        if (eq && eq_seen + __popc(beq & ((1u << lane) - 1u)) < want) keep = true;
+        eq_seen += __popc(beq);
         const uint32_t bal = __ballot_sync(0xffffffffu, keep);
         if (lane == 0) out_bits[c / 32] = bal;
         if (keep) out_idx[total + __popc(bal & ((1u << lane) - 1u))] = j;
