@@ -191,6 +191,8 @@ int rapid3_create(rapid3_ctx** out, const rapid3_shape* shape) {
     g.N = shape->n_text + shape->n_image;
     g.nb = (g.N + 63) / 64;
     g.n_text_blocks = (shape->n_text + 63) / 64;
+    // a 128 x 128 token grid after a block-aligned text prefix: one grid row = two blocks
+    g.pair_stride = (shape->n_image == 128 * 128 && shape->n_text % 64 == 0) ? 2 : 1;
     g.stride_b = shape->stride_b;
     g.stride_h = shape->stride_h;
     g.stride_n = shape->stride_n;

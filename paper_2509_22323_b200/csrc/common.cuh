@@ -24,6 +24,7 @@ struct ImgList {
 
 struct TensorGeom {
     int H, D, N, nb, n_text_blocks;
+    int pair_stride;                          // 1 or 2: which query blocks share an attention tile
     long long stride_b, stride_h, stride_n;   // elements
 };
 

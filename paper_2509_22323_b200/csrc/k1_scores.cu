@@ -168,6 +168,7 @@ extern "C" int rapid3_block_scores_static(const rapid3_shape* s, const void* q, 
     g.N = (int)N;
     g.nb = (int)((N + 63) / 64);
     g.n_text_blocks = (s->n_text + 63) / 64;
+    g.pair_stride = 1;
     g.stride_b = s->stride_b;
     g.stride_h = s->stride_h;
     g.stride_n = s->stride_n;
