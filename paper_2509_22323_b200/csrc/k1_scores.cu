@@ -1,7 +1,7 @@
 // K1: pooled block scores.
-//   pool_kernel   : one CTA per (Q|K, image, head, 64-token block); 128-bit coalesced loads,
-//                   fp64 accumulation (the sum of <= 64 bf16 values is exact in fp64), mean over
-//                   the valid tokens of the block.  HBM-bound: reads Q and K exactly once.
+//   pool_kernel   : one warp per (Q|K, image, head, 64-token block); 128-bit coalesced loads,
+//                   fp64 accumulation, mean over the valid tokens of the block.
+//                   HBM-bound: reads Q and K exactly once.
 //   scores_kernel : S[i][j] = Qbar[i,:] . Kbar[j,:] in fp64, rounded once to fp32.
 #include "common.cuh"
 
@@ -10,49 +10,59 @@ namespace {
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
+// One warp per (Q|K, image, head, 64-token block).  A token row of D channels is D / 8 lanes of
+// 16 bytes, so one warp-wide load covers 32 / (D / 8) rows; every lane keeps fp64 sums of its 8
+// channels over the rows it sees (eight loads in flight per lane), and the lanes that hold the
+// same channels are then added with shuffles.  No shared memory.
 template <int D>
-__global__ void __launch_bounds__(256) pool_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
+__global__ void __launch_bounds__(128) pool_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
                                                    TensorGeom g, ImgList imgs, double* __restrict__ pooled) {
-    constexpr int TPR = D / 8;          // threads per token row (8 channels = 16 bytes each)
-    constexpr int RG = 256 / TPR;       // row groups
-    constexpr int RPT = 64 / RG;        // rows per thread
-    __shared__ double red[RG][D + 1];
-
-    const int blk = blockIdx.x, h = blockIdx.y;
+    constexpr int TPR = D / 8;          // lanes per token row (8 channels = 16 bytes each)
+    constexpr int RPL = 32 / TPR;       // rows per warp-wide load
+    constexpr int ITERS = 64 / RPL;     // loads per lane
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int blk = blockIdx.x * 4 + warp, h = blockIdx.y;
+    if (blk >= g.nb) return;
     const int which = blockIdx.z / imgs.n;            // 0 = Q, 1 = K
     const int p = blockIdx.z - which * imgs.n;
     const uint16_t* base = (which ? k : q) + (long long)imgs.batch[p] * g.stride_b + (long long)h * g.stride_h;
-    const int t = threadIdx.x, c = t % TPR, rg = t / TPR;
+    const int c = lane % TPR, r0 = lane / TPR;
     const int n0 = blk * 64;
     const int valid = min(64, g.N - n0);
 
-    uint4 v[RPT];
-#pragma unroll
-    for (int r = 0; r < RPT; ++r) {
-        int row = rg + r * RG;
-        v[r] = make_uint4(0, 0, 0, 0);
-        if (row < valid)
-            v[r] = __ldg(reinterpret_cast<const uint4*>(base + (long long)(n0 + row) * g.stride_n + c * 8));
-    }
     double acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.0;
 #pragma unroll
-    for (int r = 0; r < RPT; ++r) {
-        acc[0] += (double)bf16_lo(v[r].x); acc[1] += (double)bf16_hi(v[r].x);
-        acc[2] += (double)bf16_lo(v[r].y); acc[3] += (double)bf16_hi(v[r].y);
-        acc[4] += (double)bf16_lo(v[r].z); acc[5] += (double)bf16_hi(v[r].z);
-        acc[6] += (double)bf16_lo(v[r].w); acc[7] += (double)bf16_hi(v[r].w);
+    for (int it0 = 0; it0 < ITERS; it0 += 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int row = (it0 + u) * RPL + r0;
+            v[u] = make_uint4(0, 0, 0, 0);
+            if (row < valid)
+                v[u] = __ldg(reinterpret_cast<const uint4*>(base + (long long)(n0 + row) * g.stride_n + c * 8));
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            acc[0] += (double)bf16_lo(v[u].x); acc[1] += (double)bf16_hi(v[u].x);
+            acc[2] += (double)bf16_lo(v[u].y); acc[3] += (double)bf16_hi(v[u].y);
+            acc[4] += (double)bf16_lo(v[u].z); acc[5] += (double)bf16_hi(v[u].z);
+            acc[6] += (double)bf16_lo(v[u].w); acc[7] += (double)bf16_hi(v[u].w);
+        }
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) red[rg][c * 8 + e] = acc[e];
-    __syncthreads();
-    if (t < D) {
-        double s = 0.0;
-#pragma unroll 8
-        for (int r = 0; r < RG; ++r) s += red[r][t];
-        long long o = ((((long long)which * imgs.n + p) * g.H + h) * g.nb + blk) * D + t;
-        pooled[o] = s / (double)valid;
+    for (int off = TPR; off < 32; off <<= 1)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], off);
+    if (lane < TPR) {
+        double* o = pooled + ((((long long)which * imgs.n + p) * g.H + h) * g.nb + blk) * D + c * 8;
+        const double inv = 1.0 / (double)valid;
+#pragma unroll
+        for (int e = 0; e < 8; e += 2) {
+            double2 w2 = make_double2(acc[e] * inv, acc[e + 1] * inv);
+            *reinterpret_cast<double2*>(o + e) = w2;
+        }
     }
 }
 
@@ -93,11 +103,11 @@ __global__ void __launch_bounds__(256) scores_kernel(const double* __restrict__ 
 
 cudaError_t launch_block_pool(const void* q, const void* k, const TensorGeom& g, const ImgList& imgs,
                               double* pooled, cudaStream_t s) {
-    dim3 grid(g.nb, g.H, 2 * imgs.n);
+    dim3 grid((g.nb + 3) / 4, g.H, 2 * imgs.n);
     if (g.D == 128)
-        pool_kernel<128><<<grid, 256, 0, s>>>((const uint16_t*)q, (const uint16_t*)k, g, imgs, pooled);
+        pool_kernel<128><<<grid, 128, 0, s>>>((const uint16_t*)q, (const uint16_t*)k, g, imgs, pooled);
     else
-        pool_kernel<64><<<grid, 256, 0, s>>>((const uint16_t*)q, (const uint16_t*)k, g, imgs, pooled);
+        pool_kernel<64><<<grid, 128, 0, s>>>((const uint16_t*)q, (const uint16_t*)k, g, imgs, pooled);
     return cudaGetLastError();
 }
 
