@@ -137,14 +137,14 @@ int get_map(rapid3_ctx* c, const void* base, const CUtensorMap** out) {
 int attn_launch(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out, const ImgList& l,
                 const int32_t* kept_idx, const int32_t* kept_cnt, const uint64_t* bitmask, float scale,
                 cudaStream_t st) {
-    const CUtensorMap *mq, *mk, *mv, *mo;
+    const CUtensorMap *mq, *mk, *mv;
     int r;
-    if ((r = get_map(c, q, &mq)) || (r = get_map(c, k, &mk)) || (r = get_map(c, v, &mv)) || (r = get_map(c, out, &mo)))
-        return r;
-    CUtensorMap tq = *mq, tk = *mk, tv = *mv, to = *mo;   // copies: a later get_map may recycle the slot
+    if ((r = get_map(c, q, &mq)) || (r = get_map(c, k, &mk)) || (r = get_map(c, v, &mv))) return r;
+    if (reinterpret_cast<uintptr_t>(out) % 16) return RAPID3_ERR_INVALID_ARG;
+    CUtensorMap tq = *mq, tk = *mk, tv = *mv;   // copies: a later get_map may recycle the slot
     {
         ProfScope ps(c, PROF_ATTN, st);
-        if (launch_attention(tq, tk, tv, to, c->g, l, kept_idx, kept_cnt, bitmask, scale, c->sched, c->status, st) != cudaSuccess)
+        if (launch_attention(tq, tk, tv, out, c->g, l, kept_idx, kept_cnt, bitmask, scale, c->sched, c->status, st) != cudaSuccess)
             return RAPID3_ERR_CUDA;
     }
     c->launches += 1;

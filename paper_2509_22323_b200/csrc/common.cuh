@@ -39,8 +39,7 @@ cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const I
 // K3: attention over kept tiles.  `bitmask` (optional) is the select kernel's bitmask of the same
 // lists; when present the kernel reads it instead of walking the lists.  `sched` points at two
 // ints in device memory that are zero between launches (work counter, finished-CTA counter).
-cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv,
-                             const CUtensorMap& tmo,
+cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv, void* out,
                              const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
                              const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* sched,
                              int* status, cudaStream_t s);

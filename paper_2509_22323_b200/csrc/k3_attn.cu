@@ -55,6 +55,7 @@ struct AttnParams {
     int n_dense;                   // leading images of the list that keep every block
     int n_items;                   // work items of this launch
     int* sched;                    // [0] next item, [1] CTAs that have finished (both return to 0)
+    uint16_t* out;
     int* status;
     float scale_log2;
 };
@@ -65,9 +66,8 @@ struct Cfg {
     static constexpr int QTILE_BYTES = 128 * D * 2;         // one 128-row Q tile
     static constexpr int KV_BYTES = 64 * D * 2;             // one key block of K or of V
     static constexpr int KS = (D == 128) ? 4 : 8;           // K ring stages
-    static constexpr int VS = (D == 128) ? 3 : 8;           // V ring stages
-    static constexpr int OSTAGE_BYTES = 128 * 128;          // output staging of one tile: 128 rows x one 64-channel half
-    static constexpr int DATA_BYTES = 2 * QTILE_BYTES + (KS + VS) * KV_BYTES + 2 * OSTAGE_BYTES;
+    static constexpr int VS = (D == 128) ? 4 : 8;           // V ring stages
+    static constexpr int DATA_BYTES = 2 * QTILE_BYTES + (KS + VS) * KV_BYTES;
 };
 
 // One work item as the scheduler hands it to the other warps.
@@ -87,7 +87,6 @@ struct __align__(16) Ctl {
     unsigned long long s_full[2][2], p_full[2][2];
     unsigned long long pv_done[2], o_done[2], o_empty[2], drain[2];
     unsigned long long list_full[2], list_empty[2];
-    unsigned long long ost_full[2], ost_free[2];   // output staging of a tile: written (128 threads) / read out by the store
     uint32_t tmem_base;
     volatile int abort_flag;
     uint32_t bm[4][32];
@@ -106,7 +105,7 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
-            const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo, const AttnParams prm) {
+            const __grid_constant__ CUtensorMap tmv, const AttnParams prm) {
     using C = Cfg<D>;
     constexpr int DH = C::DH, KS = C::KS, VS = C::VS;
     extern __shared__ uint8_t smem_raw[];
@@ -114,7 +113,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
     uint8_t* smem = smem_raw + pad;
     const uint32_t sQ = raw + pad, sK = sQ + 2 * C::QTILE_BYTES, sV = sK + KS * C::KV_BYTES;
-    const uint32_t sO = sV + VS * C::KV_BYTES;
     Ctl* ctl = reinterpret_cast<Ctl*>(smem + C::DATA_BYTES);
 
     const int tid = threadIdx.x, lane = tid % 32;
@@ -158,15 +156,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             mbar_init(smem_u32(&ctl->drain[t]), 1);
             mbar_init(bLF + 8 * t, 1);
             mbar_init(bLE + 8 * t, N_CONSUMER_WARPS);
-            mbar_init(smem_u32(&ctl->ost_full[t]), 128);
-            mbar_init(smem_u32(&ctl->ost_free[t]), 1);
         }
         ctl->abort_flag = 0;
         fence_mbar_init();
         prefetch_tmap(&tmq);
         prefetch_tmap(&tmk);
         prefetch_tmap(&tmv);
-        prefetch_tmap(&tmo);
     }
     if (warp == MMA_WARP0) {
         tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS);
@@ -471,8 +466,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         uint32_t r0[32], r1[32];
         int n = 0;                                     // blocks of this tile so far, over all items
         int od = 0;                                    // items in which this tile had work (phases of o_done)
-        int ost = 0;                                   // uses of the output staging buffer so far
-        const uint32_t bOS = smem_u32(&ctl->ost_full[t]), bOF = smem_u32(&ctl->ost_free[t]);
         for (int it = 0; ok; ++it) {
             const int lbuf = it & 1;
             const ItemList* L = &ctl->list[lbuf];
@@ -569,71 +562,55 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                 ++n;
             }
             if (!ok) break;
-            // epilogue: O out of TMEM (which frees it for the next item), O / l -> bf16 -> the tile's
-            // staging buffer in the tensor map's 128-byte swizzled layout -> TMA stores, one 64-channel
-            // half at a time; rows past the end of the sequence are clipped by the store.  The stores
-            // drain in the background while the warps go on with the next item.
-            const int i0 = L->i0, hh = L->h, bb = L->b;
+            // epilogue: O out of TMEM (which frees it for the next item), O / l -> bf16 -> global
+            const int n_glob = (L->i0 + a) * 64 + (row & 63);
+            uint16_t* orow = prm.out + (long long)L->b * g.stride_b + (long long)L->h * g.stride_h +
+                             (long long)n_glob * g.stride_n;
             release_list(lbuf);
             if (n_mine > 0 && !(ok = wait_warp(bOD + 8 * t, od & 1))) break;
             od += n_mine > 0;
             tc_fence_after();
             const float l_run = (l0 + l1) + (l2 + l3);
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            uint8_t* so = smem + (sO - sQ) + t * C::OSTAGE_BYTES + row * 128;
-            const bool storer = wl == 0 && lane == 0;
+            if (n_mine > 0) {
+                tmem_ld32(tO, r0);
+                tmem_ld32(tO + 32, r1);
+                tc_wait_ld();
+            } else {
 #pragma unroll
-            for (int dh = 0; dh < DH; ++dh) {
+                for (int e = 0; e < 32; ++e) r0[e] = r1[e] = 0u;
+            }
+            if (D == 64) {
+                tc_fence_before();
+                mbar_arrive(bOE + 8 * t);
+            }
+            auto store32 = [&](const uint32_t (&r)[32], int ch) {
+                if (n_glob < N) {
+#pragma unroll
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        uint4 o;
+                        o.x = pack_bf16(__uint_as_float(r[v4 * 8 + 0]) * inv, __uint_as_float(r[v4 * 8 + 1]) * inv);
+                        o.y = pack_bf16(__uint_as_float(r[v4 * 8 + 2]) * inv, __uint_as_float(r[v4 * 8 + 3]) * inv);
+                        o.z = pack_bf16(__uint_as_float(r[v4 * 8 + 4]) * inv, __uint_as_float(r[v4 * 8 + 5]) * inv);
+                        o.w = pack_bf16(__uint_as_float(r[v4 * 8 + 6]) * inv, __uint_as_float(r[v4 * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4*>(orow + ch * 32 + v4 * 8) = o;
+                    }
+                }
+            };
+            store32(r0, 0);
+            store32(r1, 1);
+            if (D == 128) {
                 if (n_mine > 0) {
-                    tmem_ld32(tO + dh * 64, r0);
-                    tmem_ld32(tO + dh * 64 + 32, r1);
+                    tmem_ld32(tO + 64, r0);
+                    tmem_ld32(tO + 96, r1);
                     tc_wait_ld();
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) r0[e] = r1[e] = 0u;
                 }
-                if (dh == DH - 1) {                     // O is in registers: the next item may overwrite it
-                    tc_fence_before();
-                    mbar_arrive(bOE + 8 * t);
-                }
-                // the previous use of the staging buffer must have been read out by its store
-                if (ost > 0) {
-                    if (storer) {
-                        bulk_wait_read_all();
-                        mbar_arrive(bOF);
-                    }
-                    if (!(ok = wait_warp(bOF, (ost - 1) & 1))) break;
-                }
-#pragma unroll
-                for (int v4 = 0; v4 < 8; ++v4) {
-                    const uint32_t* r = v4 < 4 ? r0 : r1;
-                    const int q = (v4 & 3) * 8;
-                    uint4 o;
-                    o.x = pack_bf16(__uint_as_float(r[q + 0]) * inv, __uint_as_float(r[q + 1]) * inv);
-                    o.y = pack_bf16(__uint_as_float(r[q + 2]) * inv, __uint_as_float(r[q + 3]) * inv);
-                    o.z = pack_bf16(__uint_as_float(r[q + 4]) * inv, __uint_as_float(r[q + 5]) * inv);
-                    o.w = pack_bf16(__uint_as_float(r[q + 6]) * inv, __uint_as_float(r[q + 7]) * inv);
-                    *reinterpret_cast<uint4*>(so + ((v4 ^ (row & 7)) << 4)) = o;
-                }
-                fence_proxy_async_smem();
-                mbar_arrive(bOS);
-                if (storer) {
-                    if ((ok = wait(bOS, ost & 1))) {
-#pragma unroll
-                        for (int c = 0; c < 2; ++c) {
-                            const int qa = ps2 ? 2 * c + t : 2 * t + c;
-                            if ((i0 + qa) * 64 < N)
-                                tma_store_4d(&tmo, sO + t * C::OSTAGE_BYTES + c * BLK_BYTES, dh * 64, (i0 + qa) * 64, hh, bb);
-                        }
-                        bulk_commit_group();
-                    }
-                }
-                ok = __all_sync(0xffffffffu, ok);
-                ++ost;
-                if (!ok) break;
+                tc_fence_before();
+                mbar_arrive(bOE + 8 * t);
+                store32(r0, 2);
+                store32(r1, 3);
             }
         }
-        if (wl == 0 && lane == 0) bulk_wait_read_all();     // the staging buffer must outlive its last store
     }
 
     // ---------------------------------------------------------------- teardown
@@ -680,8 +657,7 @@ cudaError_t attention_static_init() {
     return cudaSuccess;
 }
 
-cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv,
-                             const CUtensorMap& tmo,
+cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv, void* out,
                              const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
                              const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* sched,
                              int* status, cudaStream_t s) {
@@ -703,6 +679,7 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
     prm.kept_cnt = kept_cnt;
     prm.bitmask32 = reinterpret_cast<const uint32_t*>(bitmask);
     prm.words32 = 2 * ((g.nb + 63) / 64);
+    prm.out = reinterpret_cast<uint16_t*>(out);
     prm.sched = sched;
     prm.status = status;
     prm.scale_log2 = softmax_scale * 1.4426950408889634f;
@@ -712,8 +689,8 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
     prm.n_items = ((g.nb + 3) / 4) * g.H * imgs.n;
     dim3 grid(prm.n_items < n_sm ? prm.n_items : n_sm, 1, 1);   // one persistent CTA per SM
     if (g.D == 128)
-        attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, tmo, prm);
+        attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, prm);
     else
-        attn_kernel<64><<<grid, NTHREADS, attn_smem_bytes<64>(), s>>>(tmq, tmk, tmv, tmo, prm);
+        attn_kernel<64><<<grid, NTHREADS, attn_smem_bytes<64>(), s>>>(tmq, tmk, tmv, prm);
     return cudaGetLastError();
 }
