@@ -38,7 +38,6 @@ struct rapid3_ctx {
     int32_t* kept_idx = nullptr;  // [B_max][H][nb][nb]
     int32_t* kept_cnt = nullptr;  // [B_max][H][nb]
     int* status = nullptr;
-    int* sched = nullptr;         // work counters of the persistent attention kernel (zero between launches)
     // host-tensor staging of rapid3_gated_step_host (created on first use)
     void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
     EncodeTiledFn encode = nullptr;
@@ -137,14 +136,14 @@ int get_map(rapid3_ctx* c, const void* base, const CUtensorMap** out) {
 int attn_launch(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out, const ImgList& l,
                 const int32_t* kept_idx, const int32_t* kept_cnt, const uint64_t* bitmask, float scale,
                 cudaStream_t st) {
-    const CUtensorMap *mq, *mk, *mv;
+    const CUtensorMap *mq, *mk, *mv, *mo;
     int r;
-    if ((r = get_map(c, q, &mq)) || (r = get_map(c, k, &mk)) || (r = get_map(c, v, &mv))) return r;
-    if (reinterpret_cast<uintptr_t>(out) % 16) return RAPID3_ERR_INVALID_ARG;
-    CUtensorMap tq = *mq, tk = *mk, tv = *mv;   // copies: a later get_map may recycle the slot
+    if ((r = get_map(c, q, &mq)) || (r = get_map(c, k, &mk)) || (r = get_map(c, v, &mv)) || (r = get_map(c, out, &mo)))
+        return r;
+    CUtensorMap tq = *mq, tk = *mk, tv = *mv, to = *mo;   // copies: a later get_map may recycle the slot
     {
         ProfScope ps(c, PROF_ATTN, st);
-        if (launch_attention(tq, tk, tv, out, c->g, l, kept_idx, kept_cnt, bitmask, scale, c->sched, c->status, st) != cudaSuccess)
+        if (launch_attention(tq, tk, tv, to, c->g, l, kept_idx, kept_cnt, bitmask, scale, c->status, st) != cudaSuccess)
             return RAPID3_ERR_CUDA;
     }
     c->launches += 1;
@@ -215,9 +214,7 @@ int rapid3_create(rapid3_ctx** out, const rapid3_shape* shape) {
               cudaMalloc(&c->kept_idx, B * H * nb * nb * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&c->kept_cnt, B * H * nb * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&c->status, sizeof(int)) == cudaSuccess &&
-              cudaMemset(c->status, 0, sizeof(int)) == cudaSuccess &&
-              cudaMalloc(&c->sched, 2 * sizeof(int)) == cudaSuccess &&
-              cudaMemset(c->sched, 0, 2 * sizeof(int)) == cudaSuccess;
+              cudaMemset(c->status, 0, sizeof(int)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         rapid3_destroy(c);
@@ -240,7 +237,6 @@ int rapid3_destroy(rapid3_ctx* c) {
     cudaFree(c->kept_idx);
     cudaFree(c->kept_cnt);
     cudaFree(c->status);
-    cudaFree(c->sched);
     for (void* s : c->stage) cudaFree(s);
     for (auto& r : c->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     delete c;

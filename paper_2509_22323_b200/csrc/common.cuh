@@ -37,10 +37,9 @@ cudaError_t launch_block_scores(const double* pooled, const TensorGeom& g, int n
 cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const ImgList& imgs,
                                uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s);
 // K3: attention over kept tiles.  `bitmask` (optional) is the select kernel's bitmask of the same
-// lists; when present the kernel reads it instead of walking the lists.  `sched` points at two
-// ints in device memory that are zero between launches (work counter, finished-CTA counter).
-cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv, void* out,
-                             const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
-                             const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* sched,
-                             int* status, cudaStream_t s);
+// lists; when present the kernel reads it instead of walking the lists.
+cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv,
+                             const CUtensorMap& tmo, const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
+                             const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* status,
+                             cudaStream_t s);
 cudaError_t attention_static_init();

@@ -1,29 +1,24 @@
 // K3: masked flash-style joint attention over the kept key tiles (sm_100a).
 //
-// Persistent kernel: one CTA per SM takes work items from a counter in global memory until none
-// is left.  An item is (image, head, four consecutive 64-token query blocks) = two 128-row Q tiles
-// (the native UMMA M).  The four query blocks' kept lists are merged into one ascending union
-// list; the producer streams each key block of the union once through shared memory and both
-// tiles use it.  A tile issues no MMA for a key block that neither of its query blocks kept; a
-// 64x64 sub-tile whose key block is not in that query block's own list gets P = 0, so each query
-// block attends exactly its own kept set.  Items are numbered longest first (dense images and the
-// text-row quads of sparse images, then the other quads by descending keep ratio), so taking them
-// in order from the counter is longest-processing-time-first scheduling.
+// One CTA per (image, head, four adjacent 64-token query blocks) = two 128-row Q tiles (the
+// native UMMA M), one CTA per SM.  The four query blocks' ascending kept lists are merged into
+// one union list; the producer streams each key block of the union once through shared memory
+// and both tiles use it, which nearly halves the L2 -> SM traffic per MMA and leaves room for
+// deep K / V rings.  A tile issues no MMA for a key block that neither of its query blocks
+// kept; inside a tile a 64x64 sub-tile whose key block is not in that query block's own list
+// gets P = 0, so each query block attends exactly its own kept set.
 //
-// Roles (384 threads), each a loop over the CTA's items that shares nothing but mbarriers:
-//   warp 11     scheduler: takes the next item, builds its union list into one of two list
-//               buffers while the previous item is still being computed
-//   warp 8      producer: TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of the Q tiles as
-//               soon as the previous item's last Q K^T has read them, then the gathered K and V
-//               blocks through two rings of shared-memory stages that run on across items
+// Roles (352 threads):
+//   warp 8      producer: TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of Q once, then
+//               the gathered K and V blocks into two rings of shared-memory stages
 //   warps 9,10  UMMA issue, one warp per tile (warp 9 also owns the TMEM allocation).  S of a
 //               tile is double buffered in TMEM (2 x 64 fp32 columns): S(n+1) = Q K^T is issued
-//               before O += P(n) V.  Both warps walk the whole union list, K one block ahead of
-//               V; a stage is released when both have passed it
-//   warps 0-7   softmax, four warps per tile: thread = one query row; S(n) from TMEM in one pass,
-//               fp32 online softmax with lazy rescale of O, P(n) written back over S(n) as bf16;
-//               at the end of an item O / l is read out of TMEM (which frees it for the next
-//               item) and stored
+//               before O += P(n) V, so the tensor pipe works on the next scores while the
+//               softmax warps are busy with the current ones.  Both warps walk the same union
+//               list one block ahead in K than in V; a stage is released when both have passed it
+//   warps 0-7   softmax, four warps per tile: thread = one query row; S(n) from TMEM in one pass
+//               (64 registers), fp32 online softmax with lazy rescale of O, P(n) written back
+//               over S(n) as bf16, final O / l store
 // TMEM: tile t owns columns [256 t, 256 t + 256): S(n) at 64 (n & 1), O at 128.
 // Every mbarrier wait is bounded; a wait that runs out records RAPID3_ERR_TIMEOUT in the status
 // word and the CTA drains its copies, releases its TMEM and exits normally.
@@ -34,9 +29,8 @@ using namespace ptx;
 
 namespace {
 
-constexpr int NTHREADS = 384;
-constexpr int PRODUCER_WARP = 8, MMA_WARP0 = 9, SCHED_WARP = 11;
-constexpr int N_CONSUMER_WARPS = 11;   // warps that read a union list: 8 softmax, producer, 2 MMA
+constexpr int NTHREADS = 352;
+constexpr int PRODUCER_WARP = 8, MMA_WARP0 = 9;
 constexpr int TMEM_COLS = 512;
 constexpr int TILE_COLS = 256;      // TMEM columns of one Q tile
 constexpr int O_COL = 128;
@@ -53,9 +47,6 @@ struct AttnParams {
     const uint32_t* bitmask32;     // optional: the same mask as 32-bit words, [slot][H][nb][words32]
     int words32;
     int n_dense;                   // leading images of the list that keep every block
-    int n_items;                   // work items of this launch
-    int* sched;                    // [0] next item, [1] CTAs that have finished (both return to 0)
-    uint16_t* out;
     int* status;
     float scale_log2;
 };
@@ -70,27 +61,18 @@ struct Cfg {
     static constexpr int DATA_BYTES = 2 * QTILE_BYTES + (KS + VS) * KV_BYTES;
 };
 
-// One work item as the scheduler hands it to the other warps.
-struct ItemList {
-    int valid;                      // 0: no more work
-    int b, h, i0;                   // batch index, head, first query block of the quad
-    int n_u;                        // length of the union list
-    int n_tile[2];                  // key blocks each tile uses
-    int16_t u_blk[RAPID3_MAX_NB];
-    uint8_t u_flag[RAPID3_MAX_NB];  // bit a: query block a of the quad keeps this key block
-};
-
 struct __align__(16) Ctl {
-    unsigned long long q_full, q_empty[2];
+    unsigned long long q_full;
     unsigned long long k_full[MAX_STAGES], k_empty[MAX_STAGES];
     unsigned long long v_full[MAX_STAGES], v_empty[MAX_STAGES];
     unsigned long long s_full[2][2], p_full[2][2];
-    unsigned long long pv_done[2], o_done[2], o_empty[2], drain[2];
-    unsigned long long list_full[2], list_empty[2];
+    unsigned long long pv_done[2], o_done[2], drain[2];
     uint32_t tmem_base;
+    int n_u;
     volatile int abort_flag;
     uint32_t bm[4][32];
-    ItemList list[2];
+    int16_t u_blk[RAPID3_MAX_NB];
+    uint8_t u_flag[RAPID3_MAX_NB];      // bit a: query block a of the quad keeps this key block
 };
 
 template <int D>
@@ -105,7 +87,7 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 template <int D>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
-            const __grid_constant__ CUtensorMap tmv, const AttnParams prm) {
+            const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo, const AttnParams prm) {
     using C = Cfg<D>;
     constexpr int DH = C::DH, KS = C::KS, VS = C::VS;
     extern __shared__ uint8_t smem_raw[];
@@ -121,19 +103,43 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     const int warp = __shfl_sync(0xffffffffu, tid / 32, 0);
     const TensorGeom& g = prm.g;
     const int nb = g.nb, N = g.N;
+    // Work order, longest first (CTAs start in block-index order as SMs free up, so this is
+    // longest-processing-time-first scheduling): every quad of the dense images and the quads of
+    // the sparse images that hold a text query block walk all nb key blocks; the other quads of the
+    // sparse images follow, image by image in the list's order (descending keep ratio).
+    int quad, h, p;
+    {
+        const int nq = (nb + 3) >> 2, ntq = min(nq, (g.n_text_blocks + 3) >> 2);
+        const int nd = prm.n_dense, ns = prm.imgs.n - nd;
+        int L = blockIdx.x;
+        const int heavy_dense = nd * g.H * nq, heavy_sparse = ns * g.H * ntq;
+        if (L < heavy_dense) {
+            p = L / (g.H * nq); L -= p * g.H * nq;
+            h = L / nq; quad = L - h * nq;
+        } else if (L < heavy_dense + heavy_sparse) {
+            L -= heavy_dense;
+            p = L / (g.H * ntq); L -= p * g.H * ntq; p += nd;
+            h = L / ntq; quad = L - h * ntq;
+        } else {
+            L -= heavy_dense + heavy_sparse;
+            const int nl = nq - ntq;
+            p = L / (g.H * nl); L -= p * g.H * nl; p += nd;
+            h = L / nl; quad = ntq + (L - h * nl);
+        }
+    }
+    const int b = prm.imgs.batch[p], slot = prm.imgs.slot[p];
+    const int i0 = 4 * quad;
     // Which two of the quad's four query blocks form a 128-row tile: neighbours (a, a + 1), or, when
     // a row of the image grid spans two blocks, vertical neighbours (a, a + 2), whose kept lists
     // overlap far more (measured on the 128 x 128 grid at keep ratio 0.25: 90 % against 63 % of
     // the tile's MMA work lands on kept 64 x 64 sub-tiles)
     const bool ps2 = g.pair_stride == 2;
 
-    const uint32_t bQ = smem_u32(&ctl->q_full), bQE = smem_u32(&ctl->q_empty[0]);             // [tile]: + 8 t
+    const uint32_t bQ = smem_u32(&ctl->q_full);
     const uint32_t bKF = smem_u32(&ctl->k_full[0]), bKE = smem_u32(&ctl->k_empty[0]);
     const uint32_t bVF = smem_u32(&ctl->v_full[0]), bVE = smem_u32(&ctl->v_empty[0]);
     const uint32_t bSF = smem_u32(&ctl->s_full[0][0]), bPF = smem_u32(&ctl->p_full[0][0]);   // [tile][buf]: + 16 t + 8 buf
     const uint32_t bPV = smem_u32(&ctl->pv_done[0]), bOD = smem_u32(&ctl->o_done[0]);        // [tile]: + 8 t
-    const uint32_t bOE = smem_u32(&ctl->o_empty[0]);                                          // [tile]: + 8 t
-    const uint32_t bLF = smem_u32(&ctl->list_full[0]), bLE = smem_u32(&ctl->list_empty[0]);   // [buf]: + 8 buf
 
     // ---------------------------------------------------------------- setup
     if (tid == 0) {
@@ -149,28 +155,88 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             mbar_init(bPF + 8 * s, 128);
         }
         for (int t = 0; t < 2; ++t) {
-            mbar_init(bQE + 8 * t, 1);
             mbar_init(bPV + 8 * t, 1);
             mbar_init(bOD + 8 * t, 1);
-            mbar_init(bOE + 8 * t, 128);
             mbar_init(smem_u32(&ctl->drain[t]), 1);
-            mbar_init(bLF + 8 * t, 1);
-            mbar_init(bLE + 8 * t, N_CONSUMER_WARPS);
         }
         ctl->abort_flag = 0;
+        ctl->n_u = 0;
         fence_mbar_init();
         prefetch_tmap(&tmq);
         prefetch_tmap(&tmk);
         prefetch_tmap(&tmv);
+        prefetch_tmap(&tmo);
     }
+    if (tid < 128) ctl->bm[tid / 32][tid % 32] = 0;
     if (warp == MMA_WARP0) {
         tmem_alloc(smem_u32(&ctl->tmem_base), TMEM_COLS);
         tmem_relinquish();
         tc_fence_before();
     }
     __syncthreads();
+
+    // The Q tiles do not depend on the mask: start their loads before the union list is built.
+    if (warp == PRODUCER_WARP && lane == 0) {
+        mbar_arrive_expect_tx(bQ, 2 * C::QTILE_BYTES);
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int dh = 0; dh < DH; ++dh)
+                tma_load_4d(sQ + (ps2 ? (a & 1) : (a >> 1)) * C::QTILE_BYTES + dh * QHALF_BYTES +
+                                (ps2 ? (a >> 1) : (a & 1)) * BLK_BYTES, &tmq, bQ,
+                            dh * 64, (i0 + a) * 64, h, b);
+    }
+
+    // ---------------------------------------------------------------- union of the four kept lists
+    // bm[a] = bit set of the key blocks query block a keeps: copied from the bitmask when the
+    // caller has one, else rebuilt from the kept list; every block is kept for a dense image.
+    const int nw = (nb + 31) >> 5;
+    if (slot >= 0 && prm.bitmask32 != nullptr) {
+        if (tid < 4 * nw) {
+            const int a = tid / nw, w = tid - a * nw;
+            if (i0 + a < nb)
+                ctl->bm[a][w] = prm.bitmask32[(((long long)slot * g.H + h) * nb + i0 + a) * prm.words32 + w];
+        }
+    } else if (slot >= 0 && prm.kept_idx != nullptr) {
+        for (int a = 0; a < 4 && i0 + a < nb; ++a) {
+            const long long row = ((long long)slot * g.H + h) * nb + i0 + a;
+            const int cnt = min(max(prm.kept_cnt[row], 0), nb);
+            const int32_t* lst = prm.kept_idx + row * nb;
+            for (int e = tid; e < cnt; e += NTHREADS) {
+                const int j = lst[e];
+                if ((unsigned)j < (unsigned)nb) atomicOr(&ctl->bm[a][j >> 5], 1u << (j & 31));
+                else atomicExch(prm.status, RAPID3_ERR_BAD_LIST);
+            }
+        }
+    } else if (tid < 32) {
+        const int n = min(max(nb - tid * 32, 0), 32);
+        const uint32_t val = n == 32 ? 0xffffffffu : ((1u << n) - 1u);
+        for (int a = 0; a < 4; ++a) ctl->bm[a][tid] = (i0 + a < nb) ? val : 0u;
+    }
+    __syncthreads();
+    // one thread per key block: its position in the ascending union list is the number of union
+    // bits below it
+    for (int j = tid; j < nb; j += NTHREADS) {
+        const int w = j >> 5, bit = j & 31;
+        const uint32_t m0 = ctl->bm[0][w], m1 = ctl->bm[1][w], m2 = ctl->bm[2][w], m3 = ctl->bm[3][w];
+        const uint32_t u = m0 | m1 | m2 | m3;
+        if ((u >> bit) & 1u) {
+            int pos = __popc(u & ((1u << bit) - 1u));
+            for (int x = 0; x < w; ++x) pos += __popc(ctl->bm[0][x] | ctl->bm[1][x] | ctl->bm[2][x] | ctl->bm[3][x]);
+            ctl->u_blk[pos] = (int16_t)j;
+            ctl->u_flag[pos] = (uint8_t)(((m0 >> bit) & 1u) | (((m1 >> bit) & 1u) << 1) | (((m2 >> bit) & 1u) << 2) |
+                                         (((m3 >> bit) & 1u) << 3));
+        }
+    }
+    if (tid == 0) {
+        int tot = 0;
+        for (int x = 0; x < nw; ++x) tot += __popc(ctl->bm[0][x] | ctl->bm[1][x] | ctl->bm[2][x] | ctl->bm[3][x]);
+        ctl->n_u = tot;
+    }
+    __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    const int n_u = ctl->n_u;
 
     auto fail = [&]() {
         atomicExch(prm.status, RAPID3_ERR_TIMEOUT);
@@ -189,180 +255,52 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     auto wait_warp = [&](uint32_t bar, uint32_t parity) -> bool {
         return __all_sync(0xffffffffu, wait(bar, parity));
     };
-    // a consumer warp is done with list buffer `buf`
-    auto release_list = [&](int buf) {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bLE + 8 * buf);
-    };
 
-    if (warp == SCHED_WARP) {
-        // ------------------------------------------------------------ scheduler
-        const int nq = (nb + 3) >> 2, ntq = min(nq, (g.n_text_blocks + 3) >> 2);
-        const int nd = prm.n_dense, ns = prm.imgs.n - nd;
-        const int heavy_dense = nd * g.H * nq, heavy_sparse = ns * g.H * ntq;
-        const int nw = (nb + 31) >> 5;
-        for (int it = 0;; ++it) {
-            const int buf = it & 1;
-            ItemList* L = &ctl->list[buf];
-            if (it >= 2 && !wait_warp(bLE + 8 * buf, ((it >> 1) & 1) ^ 1)) break;
-            int item = 0;
-            if (lane == 0) item = atomicAdd(prm.sched, 1);
-            item = __shfl_sync(0xffffffffu, item, 0);
-            if (item >= prm.n_items) {
-                if (lane == 0) {
-                    L->valid = 0;
-                    mbar_arrive(bLF + 8 * buf);
-                }
-                break;
-            }
-            // items are numbered longest first: every quad of the dense images, the quads of the
-            // sparse images that hold a text query block (they walk all nb key blocks), then the
-            // other quads of the sparse images in the list's order (descending keep ratio)
-            int quad, h, p, x = item;
-            if (x < heavy_dense) {
-                p = x / (g.H * nq); x -= p * g.H * nq;
-                h = x / nq; quad = x - h * nq;
-            } else if (x < heavy_dense + heavy_sparse) {
-                x -= heavy_dense;
-                p = x / (g.H * ntq); x -= p * g.H * ntq; p += nd;
-                h = x / ntq; quad = x - h * ntq;
-            } else {
-                x -= heavy_dense + heavy_sparse;
-                const int nl = nq - ntq;
-                p = x / (g.H * nl); x -= p * g.H * nl; p += nd;
-                h = x / nl; quad = ntq + (x - h * nl);
-            }
-            const int slot = prm.imgs.slot[p], i0 = 4 * quad;
-            // bm[a] = bit set of the key blocks query block a keeps: copied from the bitmask when the
-            // caller has one, else rebuilt from the kept list; every block for a dense image
-            for (int a = 0; a < 4; ++a) ctl->bm[a][lane] = 0u;
-            __syncwarp();
-            if (slot >= 0 && prm.bitmask32 != nullptr) {
-                for (int a = 0; a < 4 && i0 + a < nb; ++a)
-                    if (lane < nw)
-                        ctl->bm[a][lane] = prm.bitmask32[(((long long)slot * g.H + h) * nb + i0 + a) * prm.words32 + lane];
-            } else if (slot >= 0 && prm.kept_idx != nullptr) {
-                for (int a = 0; a < 4 && i0 + a < nb; ++a) {
-                    const long long row = ((long long)slot * g.H + h) * nb + i0 + a;
-                    const int cnt = min(max(prm.kept_cnt[row], 0), nb);
-                    const int32_t* lst = prm.kept_idx + row * nb;
-                    for (int e = lane; e < cnt; e += 32) {
-                        const int j = lst[e];
-                        if ((unsigned)j < (unsigned)nb) atomicOr(&ctl->bm[a][j >> 5], 1u << (j & 31));
-                        else atomicExch(prm.status, RAPID3_ERR_BAD_LIST);
-                    }
-                }
-            } else {
-                const int n = min(max(nb - lane * 32, 0), 32);
-                const uint32_t val = n == 32 ? 0xffffffffu : ((1u << n) - 1u);
-                for (int a = 0; a < 4; ++a) ctl->bm[a][lane] = (i0 + a < nb) ? val : 0u;
-            }
-            __syncwarp();
-            // lane w owns union word w: its position base is the number of union bits in lower words
-            const uint32_t m0 = ctl->bm[0][lane], m1 = ctl->bm[1][lane], m2 = ctl->bm[2][lane], m3 = ctl->bm[3][lane];
-            uint32_t u = m0 | m1 | m2 | m3;
-            const uint32_t tb0 = ps2 ? 5u : 3u, tb1 = ps2 ? 10u : 12u;
-            const int c = __popc(u);
-            int incl = c;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            int pos = incl - c, nt0 = 0, nt1 = 0;
-            while (u) {
-                const int bit = __ffs(u) - 1;
-                u &= u - 1;
-                const uint32_t f = ((m0 >> bit) & 1u) | (((m1 >> bit) & 1u) << 1) | (((m2 >> bit) & 1u) << 2) |
-                                   (((m3 >> bit) & 1u) << 3);
-                L->u_blk[pos] = (int16_t)(lane * 32 + bit);
-                L->u_flag[pos] = (uint8_t)f;
-                nt0 += (f & tb0) != 0;
-                nt1 += (f & tb1) != 0;
-                ++pos;
-            }
-            nt0 = __reduce_add_sync(0xffffffffu, nt0);
-            nt1 = __reduce_add_sync(0xffffffffu, nt1);
-            if (lane == 31) {
-                L->valid = 1;
-                L->b = prm.imgs.batch[p];
-                L->h = h;
-                L->i0 = i0;
-                L->n_u = incl;
-                L->n_tile[0] = nt0;
-                L->n_tile[1] = nt1;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bLF + 8 * buf);
-        }
-    } else if (warp == PRODUCER_WARP) {
+    if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ producer
-        int kc = 0, vc = 0;                 // key blocks of K / of V issued so far, over all items
-        bool q_pending = false;
-        bool ok = true;
-        for (int it = 0; ok; ++it) {
-            const int buf = it & 1;
-            const ItemList* L = &ctl->list[buf];
-            if (!(ok = wait_warp(bLF + 8 * buf, (it >> 1) & 1))) break;
-            if (!L->valid) break;
-            const int n_u = L->n_u, h = L->h, b = L->b, i0 = L->i0;
-            if (lane == 0) {
-                // the Q buffers are free once the previous item's last Q K^T of each tile has read them
-                // (not before the first item: a tile without work arrives there at once, and a wait for
-                // "the phase before the first" is only safe while nobody has arrived yet)
-                ok = it == 0 || (wait(bQE, (it & 1) ^ 1) && wait(bQE + 8, (it & 1) ^ 1));
-                if (ok) {
-                    mbar_arrive_expect_tx(bQ, 2 * C::QTILE_BYTES);
-                    q_pending = true;
+        if (lane == 0) {
+            int k_issued = 0, v_issued = 0;
+            auto load_k = [&](int j) -> bool {
+                const int s = j % KS;
+                if (!wait(bKE + 8 * s, ((j / KS) & 1) ^ 1)) return false;
+                mbar_arrive_expect_tx(bKF + 8 * s, C::KV_BYTES);
+                const int blk = ctl->u_blk[j];
 #pragma unroll
-                    for (int a = 0; a < 4; ++a)
+                for (int dh = 0; dh < DH; ++dh)
+                    tma_load_4d(sK + s * C::KV_BYTES + dh * BLK_BYTES, &tmk, bKF + 8 * s, dh * 64, blk * 64, h, b);
+                k_issued = j + 1;
+                return true;
+            };
+            auto load_v = [&](int j) -> bool {
+                const int s = j % VS;
+                if (!wait(bVE + 8 * s, ((j / VS) & 1) ^ 1)) return false;
+                mbar_arrive_expect_tx(bVF + 8 * s, C::KV_BYTES);
+                const int blk = ctl->u_blk[j];
 #pragma unroll
-                        for (int dh = 0; dh < DH; ++dh)
-                            tma_load_4d(sQ + (ps2 ? (a & 1) : (a >> 1)) * C::QTILE_BYTES + dh * QHALF_BYTES +
-                                            (ps2 ? (a >> 1) : (a & 1)) * BLK_BYTES, &tmq, bQ, dh * 64, (i0 + a) * 64, h, b);
-                }
-                auto load_k = [&](int j) -> bool {
-                    const int s = kc % KS;
-                    if (!wait(bKE + 8 * s, ((kc / KS) & 1) ^ 1)) return false;
-                    mbar_arrive_expect_tx(bKF + 8 * s, C::KV_BYTES);
-                    const int blk = L->u_blk[j];
-#pragma unroll
-                    for (int dh = 0; dh < DH; ++dh)
-                        tma_load_4d(sK + s * C::KV_BYTES + dh * BLK_BYTES, &tmk, bKF + 8 * s, dh * 64, blk * 64, h, b);
-                    ++kc;
-                    return true;
-                };
-                auto load_v = [&](int j) -> bool {
-                    const int s = vc % VS;
-                    if (!wait(bVE + 8 * s, ((vc / VS) & 1) ^ 1)) return false;
-                    mbar_arrive_expect_tx(bVF + 8 * s, C::KV_BYTES);
-                    const int blk = L->u_blk[j];
-#pragma unroll
-                    for (int dh = 0; dh < DH; ++dh)
-                        tma_load_4d(sV + s * C::KV_BYTES + dh * BLK_BYTES, &tmv, bVF + 8 * s, dh * 64, blk * 64, h, b);
-                    ++vc;
-                    return true;
-                };
-                // K runs one block ahead of V, the order in which the MMA warps consume them
-                if (ok && n_u > 0) ok = load_k(0);
-                for (int j = 0; ok && j < n_u; ++j) {
-                    if (j + 1 < n_u && !(ok = load_k(j + 1))) break;
-                    ok = load_v(j);
-                }
+                for (int dh = 0; dh < DH; ++dh)
+                    tma_load_4d(sV + s * C::KV_BYTES + dh * BLK_BYTES, &tmv, bVF + 8 * s, dh * 64, blk * 64, h, b);
+                v_issued = j + 1;
+                return true;
+            };
+            // K runs one block ahead of V, the order in which the MMA warps consume them
+            bool ok = n_u > 0 ? load_k(0) : true;
+            for (int j = 0; ok && j < n_u; ++j) {
+                if (j + 1 < n_u && !(ok = load_k(j + 1))) break;
+                ok = load_v(j);
             }
-            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-            release_list(buf);
-        }
-        if (lane == 0 && ctl->abort_flag) {
-            // drain: do not leave the CTA while bulk copies may still land in its shared memory
-            if (q_pending) mbar_wait(bQ, 0, 1u << 18), mbar_wait(bQ, 1, 1u << 18);
-            for (int j = max(0, kc - KS); j < kc; ++j) mbar_wait(bKF + 8 * (j % KS), (j / KS) & 1, 1u << 20);
-            for (int j = max(0, vc - VS); j < vc; ++j) mbar_wait(bVF + 8 * (j % VS), (j / VS) & 1, 1u << 20);
+            if (ctl->abort_flag) {
+                // drain: do not leave the CTA while bulk copies may still land in its shared memory
+                mbar_wait(bQ, 0, 1u << 20);
+                for (int j = max(0, k_issued - KS); j < k_issued; ++j)
+                    mbar_wait(bKF + 8 * (j % KS), (j / KS) & 1, 1u << 20);
+                for (int j = max(0, v_issued - VS); j < v_issued; ++j)
+                    mbar_wait(bVF + 8 * (j % VS), (j / VS) & 1, 1u << 20);
+            }
         }
         __syncwarp();
     } else if (warp >= MMA_WARP0) {
         // ------------------------------------------------------------ UMMA issue, one warp per tile
-        // The whole warp runs the loops converged (addresses and descriptors stay warp-uniform);
+        // The whole warp runs the loop converged (addresses and descriptors stay warp-uniform);
         // one elected lane issues the tcgen05 instructions.  Both warps pass over every block of
         // the union list, K one block ahead of V, also over blocks their tile does not use: the
         // stage barriers then see every phase in order and a stage is refilled only after both
@@ -376,81 +314,62 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         const uint32_t bSFt = bSF + 16 * t, bPFt = bPF + 16 * t;
         constexpr uint32_t idesc_qk = idesc_bf16(128, 64, 0, 0);
         constexpr uint32_t idesc_pv = idesc_bf16(128, D, 0, 1);
-        int kc = 0, vc = 0;                 // key blocks of K / of V passed so far, over all items
-        int n_qk = 0, n_pv = 0;             // blocks of this tile issued so far, over all items
-        bool ok = true;
-        for (int it = 0; ok; ++it) {
-            const int buf = it & 1;
-            const ItemList* L = &ctl->list[buf];
-            if (!(ok = wait_warp(bLF + 8 * buf, (it >> 1) & 1))) break;
-            if (!L->valid) break;
-            const int n_u = L->n_u, n_mine = L->n_tile[t];
-            int qk_item = 0, pv_item = 0;   // blocks of this tile issued in this item
-            auto k_step = [&](int j) -> bool {
-                const int s = kc % KS;
-                const bool use = L->u_flag[j] & tile_bits;
-                if (!(wait_warp(bKF + 8 * s, (kc / KS) & 1))) return false;
-                ++kc;
-                if (use) {
-                    tc_fence_after();
-                    const uint32_t tS = tbase + 64 * (n_qk & 1);
-                    const uint32_t kb = sK + s * C::KV_BYTES;
-                    ++qk_item;
-                    if (leader) {
+        int n_qk = 0, n_pv = 0;                        // blocks of this tile issued so far
+        auto k_step = [&](int j) -> bool {
+            const int s = j % KS;
+            const bool use = ctl->u_flag[j] & tile_bits;
+            if (!(wait_warp(bKF + 8 * s, (j / KS) & 1))) return false;
+            if (use) {
+                tc_fence_after();
+                const uint32_t tS = tbase + 64 * (n_qk & 1);
+                const uint32_t kb = sK + s * C::KV_BYTES;
+                if (leader) {
 #pragma unroll
-                        for (int ks = 0; ks < D / 16; ++ks)
-                            mma_ss(tS, smem_desc_sw128(qb + (ks / 4) * QHALF_BYTES + (ks % 4) * 32, 16, 1024),
-                                   smem_desc_sw128(kb + (ks / 4) * BLK_BYTES + (ks % 4) * 32, 16, 1024), idesc_qk, ks > 0);
-                        tc_commit(bKE + 8 * s);
-                        tc_commit(bSFt + 8 * (n_qk & 1));
-                        if (qk_item == n_mine) tc_commit(bQE + 8 * t);   // the Q tile may be replaced
-                    }
-                    ++n_qk;
-                } else if (leader) {
-                    mbar_arrive(bKE + 8 * s);
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        mma_ss(tS, smem_desc_sw128(qb + (ks / 4) * QHALF_BYTES + (ks % 4) * 32, 16, 1024),
+                               smem_desc_sw128(kb + (ks / 4) * BLK_BYTES + (ks % 4) * 32, 16, 1024), idesc_qk, ks > 0);
+                    tc_commit(bKE + 8 * s);
+                    tc_commit(bSFt + 8 * (n_qk & 1));
                 }
-                __syncwarp();
-                return true;
-            };
-            if (!(ok = wait_warp(bQ, it & 1))) break;
-            // a tile without work frees Q at once -- but only now, after the producer has passed its own
-            // wait for the previous item's release (an earlier arrival could run a phase ahead of it)
-            if (n_mine == 0 && leader) mbar_arrive(bQE + 8 * t);
-            if (n_u > 0) ok = k_step(0);
-            for (int j = 0; ok && j < n_u; ++j) {
-                // S(n+1) reuses the buffer of P(n-1); the MMAs of the issuing thread execute in issue
-                // order, so it is written only after P(n-1) V has read it
-                if (j + 1 < n_u && !(ok = k_step(j + 1))) break;
-                const int s = vc % VS;
-                const bool use = L->u_flag[j] & tile_bits;
-                if (use && pv_item == 0 && it > 0 && !(ok = wait_warp(bOE + 8 * t, (it & 1) ^ 1))) break;   // O read out
-                if (use && !(ok = (wait_warp(bPFt + 8 * (n_pv & 1), (n_pv >> 1) & 1)))) break;
-                if (!(ok = (wait_warp(bVF + 8 * s, (vc / VS) & 1)))) break;
-                ++vc;
-                if (use) {
-                    tc_fence_after();
-                    const uint32_t tP = tbase + 64 * (n_pv & 1);
-                    const uint32_t vb = sV + s * C::KV_BYTES;
-                    ++pv_item;
-                    if (leader) {
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            mma_ts(tO, tP + ks * 8, smem_desc_sw128(vb + ks * 2048, BLK_BYTES, 1024), idesc_pv,
-                                   (pv_item > 1 || ks > 0) ? 1u : 0u);
-                        tc_commit(bVE + 8 * s);
-                        // pv_done advances one phase per block of the tile (the rescale path waits on the
-                        // previous block's phase); the item's last block also completes o_done
-                        tc_commit(bPV + 8 * t);
-                        if (pv_item == n_mine) tc_commit(bOD + 8 * t);
-                    }
-                    ++n_pv;
-                } else if (leader) {
-                    mbar_arrive(bVE + 8 * s);
-                }
-                __syncwarp();
+                ++n_qk;
+            } else if (leader) {
+                mbar_arrive(bKE + 8 * s);
             }
-            release_list(buf);
+            __syncwarp();
+            return true;
+        };
+        bool ok = (wait_warp(bQ, 0));
+        if (ok && n_u > 0) ok = k_step(0);
+        for (int j = 0; ok && j < n_u; ++j) {
+            // S(n+1) reuses the buffer of P(n-1); the MMAs of the issuing thread execute in issue
+            // order, so it is written only after P(n-1) V has read it
+            if (j + 1 < n_u && !(ok = k_step(j + 1))) break;
+            const int s = j % VS;
+            const bool use = ctl->u_flag[j] & tile_bits;
+            if (use && !(ok = (wait_warp(bPFt + 8 * (n_pv & 1), (n_pv >> 1) & 1)))) break;
+            if (!(ok = (wait_warp(bVF + 8 * s, (j / VS) & 1)))) break;
+            if (use) {
+                tc_fence_after();
+                const uint32_t tP = tbase + 64 * (n_pv & 1);
+                const uint32_t vb = sV + s * C::KV_BYTES;
+                if (leader) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_ts(tO, tP + ks * 8, smem_desc_sw128(vb + ks * 2048, BLK_BYTES, 1024), idesc_pv,
+                               (n_pv > 0 || ks > 0) ? 1u : 0u);
+                    tc_commit(bVE + 8 * s);
+                    // pv_done advances one phase per block of the tile (the rescale path waits on the
+                    // previous block's phase); the epilogue may lag, so it has its own barrier
+                    tc_commit(bPV + 8 * t);
+                }
+                ++n_pv;
+            } else if (leader) {
+                mbar_arrive(bVE + 8 * s);
+            }
+            __syncwarp();
         }
+        if (ok && leader && n_pv > 0) tc_commit(bOD + 8 * t);
+        __syncwarp();
     } else {
         // ------------------------------------------------------------ softmax / correction / epilogue
         const int t = warp >> 2, wl = warp & 3;        // tile, lane quarter of the tile
@@ -462,161 +381,146 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         const uint32_t bSFt = bSF + 16 * t, bPFt = bPF + 16 * t, bPVt = bPV + 8 * t;
         const float c2 = prm.scale_log2;
         const int tail_valid = N - (nb - 1) * 64;      // valid tokens of the last block (1..64)
+        float m_run = -INFINITY;
+        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
         bool ok = true;
         uint32_t r0[32], r1[32];
-        int n = 0;                                     // blocks of this tile so far, over all items
-        int od = 0;                                    // items in which this tile had work (phases of o_done)
-        for (int it = 0; ok; ++it) {
-            const int lbuf = it & 1;
-            const ItemList* L = &ctl->list[lbuf];
-            if (!(ok = wait_warp(bLF + 8 * lbuf, (it >> 1) & 1))) break;
-            if (!L->valid) break;
-            const int n_u = L->n_u, n_mine = L->n_tile[t];
-            float m_run = -INFINITY;
-            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-            for (int j = 0; j < n_u; ++j) {
-                const uint32_t f = L->u_flag[j];
-                if (!(f & tile_bits)) continue;            // neither query block of the tile kept it
-                const int blk = L->u_blk[j];
-                const bool act = (f >> a) & 1u;
-                const int valid = (blk == nb - 1) ? tail_valid : 64;
-                const int buf = n & 1;
-                const uint32_t tS = lane_addr + 64 * buf;
-                if (!(ok = wait_warp(bSFt + 8 * buf, (n >> 1) & 1))) break;
-                tc_fence_after();
-                if (act) {
-                    tmem_ld32(tS, r0);
-                    tmem_ld32(tS + 32, r1);
-                    tc_wait_ld();
-                    if (valid != 64) {
+        int n = 0;                                     // blocks of this tile so far
+        for (int j = 0; j < n_u; ++j) {
+            const uint32_t f = ctl->u_flag[j];
+            if (!(f & tile_bits)) continue;            // neither query block of the tile kept it
+            const int blk = ctl->u_blk[j];
+            const bool act = (f >> a) & 1u;
+            const int valid = (blk == nb - 1) ? tail_valid : 64;
+            const int buf = n & 1;
+            const uint32_t tS = lane_addr + 64 * buf;
+            if (!(ok = wait_warp(bSFt + 8 * buf, (n >> 1) & 1))) break;
+            tc_fence_after();
+            if (act) {
+                tmem_ld32(tS, r0);
+                tmem_ld32(tS + 32, r1);
+                tc_wait_ld();
+                if (valid != 64) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            if (e >= valid) r0[e] = 0xff800000u;          // -inf: outside the sequence
-                            if (32 + e >= valid) r1[e] = 0xff800000u;
-                        }
+                    for (int e = 0; e < 32; ++e) {
+                        if (e >= valid) r0[e] = 0xff800000u;          // -inf: outside the sequence
+                        if (32 + e >= valid) r1[e] = 0xff800000u;
                     }
-                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        mx0 = max3(mx0, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]));
-                        mx1 = max3(mx1, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]));
-                        mx2 = max3(mx2, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]));
-                        mx3 = max3(mx3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]));
-                    }
-                    const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                    // lazy rescale: move the reference maximum only when it grew by more than 2^8
-                    const float m_new = fmaxf(m_run, mx);
-                    const bool grow = (m_new - m_run) * c2 > RESCALE_LOG2;    // true from -inf
-                    const bool fix_o = grow && m_run != -INFINITY;            // O holds something to rescale
-                    if (__any_sync(0xffffffffu, fix_o)) {
-                        // O must be at rest: wait for P(n-1) V
-                        if (!(ok = wait_warp(bPVt, (n - 1) & 1))) break;
-                        tc_fence_after();
-                        const float alpha = fix_o ? ex2((m_run - m_new) * c2) : 1.f;
-                        l0 *= alpha; l1 *= alpha; l2 *= alpha; l3 *= alpha;
-                        uint32_t o[32];
-#pragma unroll
-                        for (int ch = 0; ch < D / 32; ++ch) {
-                            tmem_ld32(tO + ch * 32, o);
-                            tc_wait_ld();
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                            tmem_st32(tO + ch * 32, o);
-                        }
-                    }
-                    if (grow) m_run = m_new;
-                    const float ms = m_run * c2;
-                    uint32_t pk[32];
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        float x0, x1, x2, x3;
-                        fma2(x0, x1, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]), c2, -ms);
-                        fma2(x2, x3, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]), c2, -ms);
-                        x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
-                        add2(l0, l1, x0, x1);
-                        add2(l2, l3, x2, x3);
-                        pk[e / 2] = pack_bf16(x0, x1);
-                        pk[e / 2 + 1] = pack_bf16(x2, x3);
-                    }
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        float x0, x1, x2, x3;
-                        fma2(x0, x1, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]), c2, -ms);
-                        fma2(x2, x3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]), c2, -ms);
-                        x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
-                        add2(l0, l1, x0, x1);
-                        add2(l2, l3, x2, x3);
-                        pk[16 + e / 2] = pack_bf16(x0, x1);
-                        pk[16 + e / 2 + 1] = pack_bf16(x2, x3);
-                    }
-                    tmem_st32(tS, pk);
-                } else {
-                    uint32_t z[32];
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) z[e] = 0u;
-                    tmem_st32(tS, z);
                 }
-                tc_wait_st();
-                tc_fence_before();
-                mbar_arrive(bPFt + 8 * buf);
-                ++n;
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    mx0 = max3(mx0, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]));
+                    mx1 = max3(mx1, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]));
+                    mx2 = max3(mx2, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]));
+                    mx3 = max3(mx3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]));
+                }
+                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                // lazy rescale: move the reference maximum only when it grew by more than 2^8
+                const float m_new = fmaxf(m_run, mx);
+                const bool grow = (m_new - m_run) * c2 > RESCALE_LOG2;    // true from -inf
+                const bool fix_o = grow && m_run != -INFINITY;            // O holds something to rescale
+                if (__any_sync(0xffffffffu, fix_o)) {
+                    // O must be at rest: wait for P(n-1) V
+                    if (!(ok = wait_warp(bPVt, (n - 1) & 1))) break;
+                    tc_fence_after();
+                    const float alpha = fix_o ? ex2((m_run - m_new) * c2) : 1.f;
+                    l0 *= alpha; l1 *= alpha; l2 *= alpha; l3 *= alpha;
+                    uint32_t o[32];
+#pragma unroll
+                    for (int ch = 0; ch < D / 32; ++ch) {
+                        tmem_ld32(tO + ch * 32, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tmem_st32(tO + ch * 32, o);
+                    }
+                }
+                if (grow) m_run = m_new;
+                const float ms = m_run * c2;
+                uint32_t pk[32];
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    float x0, x1, x2, x3;
+                    fma2(x0, x1, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]), c2, -ms);
+                    fma2(x2, x3, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]), c2, -ms);
+                    x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
+                    add2(l0, l1, x0, x1);
+                    add2(l2, l3, x2, x3);
+                    pk[e / 2] = pack_bf16(x0, x1);
+                    pk[e / 2 + 1] = pack_bf16(x2, x3);
+                }
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    float x0, x1, x2, x3;
+                    fma2(x0, x1, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]), c2, -ms);
+                    fma2(x2, x3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]), c2, -ms);
+                    x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
+                    add2(l0, l1, x0, x1);
+                    add2(l2, l3, x2, x3);
+                    pk[16 + e / 2] = pack_bf16(x0, x1);
+                    pk[16 + e / 2 + 1] = pack_bf16(x2, x3);
+                }
+                tmem_st32(tS, pk);
+            } else {
+                uint32_t z[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) z[e] = 0u;
+                tmem_st32(tS, z);
             }
-            if (!ok) break;
-            // epilogue: O out of TMEM (which frees it for the next item), O / l -> bf16 -> global
-            const int n_glob = (L->i0 + a) * 64 + (row & 63);
-            uint16_t* orow = prm.out + (long long)L->b * g.stride_b + (long long)L->h * g.stride_h +
-                             (long long)n_glob * g.stride_n;
-            release_list(lbuf);
-            if (n_mine > 0 && !(ok = wait_warp(bOD + 8 * t, od & 1))) break;
-            od += n_mine > 0;
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(bPFt + 8 * buf);
+            ++n;
+        }
+        // epilogue: O / l -> bf16 -> the tile's (now unused) Q buffer in the 128-byte swizzled layout
+        // of the tensor map -> TMA stores, one per (query block, 64-channel half); rows past the
+        // end of the sequence are clipped by the store
+        if (ok && n > 0) ok = wait_warp(bOD + 8 * t, 0);
+        if (ok) {
             tc_fence_after();
             const float l_run = (l0 + l1) + (l2 + l3);
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            if (n_mine > 0) {
-                tmem_ld32(tO, r0);
-                tmem_ld32(tO + 32, r1);
-                tc_wait_ld();
-            } else {
+            uint8_t* so = smem + t * C::QTILE_BYTES + row * 128;
 #pragma unroll
-                for (int e = 0; e < 32; ++e) r0[e] = r1[e] = 0u;
-            }
-            if (D == 64) {
-                tc_fence_before();
-                mbar_arrive(bOE + 8 * t);
-            }
-            auto store32 = [&](const uint32_t (&r)[32], int ch) {
-                if (n_glob < N) {
-#pragma unroll
-                    for (int v4 = 0; v4 < 4; ++v4) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(r[v4 * 8 + 0]) * inv, __uint_as_float(r[v4 * 8 + 1]) * inv);
-                        o.y = pack_bf16(__uint_as_float(r[v4 * 8 + 2]) * inv, __uint_as_float(r[v4 * 8 + 3]) * inv);
-                        o.z = pack_bf16(__uint_as_float(r[v4 * 8 + 4]) * inv, __uint_as_float(r[v4 * 8 + 5]) * inv);
-                        o.w = pack_bf16(__uint_as_float(r[v4 * 8 + 6]) * inv, __uint_as_float(r[v4 * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(orow + ch * 32 + v4 * 8) = o;
-                    }
-                }
-            };
-            store32(r0, 0);
-            store32(r1, 1);
-            if (D == 128) {
-                if (n_mine > 0) {
-                    tmem_ld32(tO + 64, r0);
-                    tmem_ld32(tO + 96, r1);
+            for (int ch = 0; ch < D / 32; ++ch) {
+                if (n > 0) {
+                    tmem_ld32(tO + ch * 32, r0);
                     tc_wait_ld();
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) r0[e] = 0u;
                 }
-                tc_fence_before();
-                mbar_arrive(bOE + 8 * t);
-                store32(r0, 2);
-                store32(r1, 3);
+#pragma unroll
+                for (int v4 = 0; v4 < 4; ++v4) {
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(r0[v4 * 8 + 0]) * inv, __uint_as_float(r0[v4 * 8 + 1]) * inv);
+                    o.y = pack_bf16(__uint_as_float(r0[v4 * 8 + 2]) * inv, __uint_as_float(r0[v4 * 8 + 3]) * inv);
+                    o.z = pack_bf16(__uint_as_float(r0[v4 * 8 + 4]) * inv, __uint_as_float(r0[v4 * 8 + 5]) * inv);
+                    o.w = pack_bf16(__uint_as_float(r0[v4 * 8 + 6]) * inv, __uint_as_float(r0[v4 * 8 + 7]) * inv);
+                    const int chunk = (ch & 1) * 4 + v4;            // 16-byte chunk of the 128-byte half row
+                    *reinterpret_cast<uint4*>(so + (ch >> 1) * QHALF_BYTES + ((chunk ^ (row & 7)) << 4)) = o;
+                }
             }
+            fence_proxy_async_smem();
+        }
+        // the two warps of a query block meet, then one lane stores the block
+        const int qb_id = a;
+        named_barrier_sync(1 + qb_id, 64);
+        if (ok && (wl & 1) == 0 && lane == 0 && (i0 + qb_id) * 64 < N) {
+#pragma unroll
+            for (int dh = 0; dh < DH; ++dh)
+                tma_store_4d(&tmo, sQ + t * C::QTILE_BYTES + dh * QHALF_BYTES + (wl >> 1) * BLK_BYTES, dh * 64,
+                             (i0 + qb_id) * 64, h, b);
+            bulk_commit_group();
+            bulk_wait_read_all();
         }
     }
 
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
-    if (warp >= MMA_WARP0 && warp < MMA_WARP0 + 2) {
+    if (warp >= MMA_WARP0) {
         if (ctl->abort_flag) {
             // make sure no UMMA of this warp is still in flight before the TMEM columns are released
             const uint32_t bT = smem_u32(&ctl->drain[warp - MMA_WARP0]);
@@ -631,15 +535,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     if (warp == MMA_WARP0) {
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
-    }
-    // the last CTA to finish puts the work counter back to zero for the next launch
-    if (tid == 0) {
-        __threadfence();
-        if (atomicAdd(prm.sched + 1, 1) == (int)gridDim.x - 1) {
-            prm.sched[0] = 0;
-            prm.sched[1] = 0;
-            __threadfence();
-        }
     }
 }
 
@@ -657,19 +552,13 @@ cudaError_t attention_static_init() {
     return cudaSuccess;
 }
 
-cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv, void* out,
+cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv,
+                             const CUtensorMap& tmo,
                              const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
-                             const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* sched,
-                             int* status, cudaStream_t s) {
+                             const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* status,
+                             cudaStream_t s) {
     if (!g_attr_set) {
         cudaError_t e = attention_static_init();
-        if (e != cudaSuccess) return e;
-    }
-    static int n_sm = 0;
-    if (n_sm == 0) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
     }
     AttnParams prm;
@@ -679,18 +568,15 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
     prm.kept_cnt = kept_cnt;
     prm.bitmask32 = reinterpret_cast<const uint32_t*>(bitmask);
     prm.words32 = 2 * ((g.nb + 63) / 64);
-    prm.out = reinterpret_cast<uint16_t*>(out);
-    prm.sched = sched;
     prm.status = status;
     prm.scale_log2 = softmax_scale * 1.4426950408889634f;
     int n_dense = 0;
     while (n_dense < imgs.n && (imgs.slot[n_dense] < 0 || kept_idx == nullptr)) ++n_dense;
     prm.n_dense = n_dense;
-    prm.n_items = ((g.nb + 3) / 4) * g.H * imgs.n;
-    dim3 grid(prm.n_items < n_sm ? prm.n_items : n_sm, 1, 1);   // one persistent CTA per SM
+    dim3 grid(((g.nb + 3) / 4) * g.H * imgs.n, 1, 1);
     if (g.D == 128)
-        attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, prm);
+        attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, tmo, prm);
     else
-        attn_kernel<64><<<grid, NTHREADS, attn_smem_bytes<64>(), s>>>(tmq, tmk, tmv, prm);
+        attn_kernel<64><<<grid, NTHREADS, attn_smem_bytes<64>(), s>>>(tmq, tmk, tmv, tmo, prm);
     return cudaGetLastError();
 }
