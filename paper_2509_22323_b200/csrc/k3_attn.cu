@@ -407,60 +407,70 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                         if (32 + e >= valid) r1[e] = 0xff800000u;
                     }
                 }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    mx0 = max3(mx0, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]));
-                    mx1 = max3(mx1, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]));
-                    mx2 = max3(mx2, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]));
-                    mx3 = max3(mx3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]));
-                }
-                const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                // lazy rescale: move the reference maximum only when it grew by more than 2^8
-                const float m_new = fmaxf(m_run, mx);
-                const bool grow = (m_new - m_run) * c2 > RESCALE_LOG2;    // true from -inf
-                const bool fix_o = grow && m_run != -INFINITY;            // O holds something to rescale
-                if (__any_sync(0xffffffffu, fix_o)) {
-                    // O must be at rest: wait for P(n-1) V
-                    if (!(ok = wait_warp(bPVt, (n - 1) & 1))) break;
-                    tc_fence_after();
-                    const float alpha = fix_o ? ex2((m_run - m_new) * c2) : 1.f;
-                    l0 *= alpha; l1 *= alpha; l2 *= alpha; l3 *= alpha;
-                    uint32_t o[32];
-#pragma unroll
-                    for (int ch = 0; ch < D / 32; ++ch) {
-                        tmem_ld32(tO + ch * 32, o);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                        tmem_st32(tO + ch * 32, o);
-                    }
-                }
-                if (grow) m_run = m_new;
-                const float ms = m_run * c2;
+                // One pass over the 64 scores gives P = 2^(S c2 - m c2) (packed to bf16), the block's
+                // partial row sums and the block's row maximum.  The pass runs with the reference
+                // maximum m as it stands, so the exponentials do not wait for this block's maximum;
+                // only when a row's maximum has grown by more than 2^8 (rare after the first blocks,
+                // always at the first block) O and l are rescaled and the pass is repeated.
                 uint32_t pk[32];
+                float b0, b1, b2, b3;
+                bool redo;
+                do {
+                    const float ms = m_run * c2;
+                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                    b0 = b1 = b2 = b3 = 0.f;
 #pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    float x0, x1, x2, x3;
-                    fma2(x0, x1, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]), c2, -ms);
-                    fma2(x2, x3, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]), c2, -ms);
-                    x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
-                    add2(l0, l1, x0, x1);
-                    add2(l2, l3, x2, x3);
-                    pk[e / 2] = pack_bf16(x0, x1);
-                    pk[e / 2 + 1] = pack_bf16(x2, x3);
-                }
+                    for (int e = 0; e < 32; e += 4) {
+                        float x0, x1, x2, x3;
+                        fma2(x0, x1, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]), c2, -ms);
+                        fma2(x2, x3, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]), c2, -ms);
+                        x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
+                        add2(b0, b1, x0, x1);
+                        add2(b2, b3, x2, x3);
+                        pk[e / 2] = pack_bf16(x0, x1);
+                        pk[e / 2 + 1] = pack_bf16(x2, x3);
+                        mx0 = max3(mx0, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]));
+                        mx1 = max3(mx1, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]));
+                    }
 #pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    float x0, x1, x2, x3;
-                    fma2(x0, x1, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]), c2, -ms);
-                    fma2(x2, x3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]), c2, -ms);
-                    x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
-                    add2(l0, l1, x0, x1);
-                    add2(l2, l3, x2, x3);
-                    pk[16 + e / 2] = pack_bf16(x0, x1);
-                    pk[16 + e / 2 + 1] = pack_bf16(x2, x3);
-                }
+                    for (int e = 0; e < 32; e += 4) {
+                        float x0, x1, x2, x3;
+                        fma2(x0, x1, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]), c2, -ms);
+                        fma2(x2, x3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]), c2, -ms);
+                        x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
+                        add2(b0, b1, x0, x1);
+                        add2(b2, b3, x2, x3);
+                        pk[16 + e / 2] = pack_bf16(x0, x1);
+                        pk[16 + e / 2 + 1] = pack_bf16(x2, x3);
+                        mx2 = max3(mx2, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]));
+                        mx3 = max3(mx3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]));
+                    }
+                    const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                    const bool grow = (mx - m_run) * c2 > RESCALE_LOG2;       // true from -inf
+                    redo = __any_sync(0xffffffffu, grow);
+                    if (redo) {
+                        const bool fix_o = grow && m_run != -INFINITY;        // O holds something to rescale
+                        if (__any_sync(0xffffffffu, fix_o)) {
+                            // O must be at rest: wait for P(n-1) V
+                            if (!(ok = wait_warp(bPVt, (n - 1) & 1))) break;
+                            tc_fence_after();
+                            const float alpha = fix_o ? ex2((m_run - mx) * c2) : 1.f;
+                            l0 *= alpha; l1 *= alpha; l2 *= alpha; l3 *= alpha;
+                            uint32_t o[32];
+#pragma unroll
+                            for (int ch = 0; ch < D / 32; ++ch) {
+                                tmem_ld32(tO + ch * 32, o);
+                                tc_wait_ld();
+#pragma unroll
+                                for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                                tmem_st32(tO + ch * 32, o);
+                            }
+                        }
+                        if (grow) m_run = mx;
+                    }
+                } while (redo);
+                if (!ok) break;
+                l0 += b0; l1 += b1; l2 += b2; l3 += b3;
                 tmem_st32(tS, pk);
             } else {
                 uint32_t z[32];
