@@ -198,3 +198,33 @@ def gated_step(Q, K, V, actions: Sequence[int], ratios: Sequence[float], n_text:
     for b, (a, r) in enumerate(zip(actions, ratios)):
         res.append(sparse_joint_attention(Q[b], K[b], V[b], n_text, r, scale) if a == 2 else None)
     return res
+
+
+# ----------------------------------------------------------------------------------------------
+# Cache-Reuse data path (paper Sec. 3.2, "Level-2: Cache-Reuse": the conditional definition of
+# O_t and the cached residual Delta = G(X) - X).  Plain numpy on bf16 bit patterns.  The paper
+# fixes no precision; the sum / difference is taken in fp32 (one IEEE rounding) and then rounded
+# to bf16 (round to nearest even), the arithmetic a bf16 pipeline has.
+
+def _bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def _f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    rounded = u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))
+    return (rounded >> np.uint32(16)).astype(np.uint16)
+
+
+def cache_step(x, o, delta, actions: Sequence[int]):
+    """x, o, delta: [B, ...] bf16 tensors (or uint16 bit arrays).  Returns (o_new, delta_new) as
+    uint16 bit arrays: action 2 (attend) refreshes delta = o - x, action 1 (reuse) sets
+    o = x + delta, action 0 (skip) leaves both as they were."""
+    xb, ob, db = (_bits(t).copy() for t in (x, o, delta))
+    for b, a in enumerate(actions):
+        xf = _bf16_bits_to_f32(xb[b])
+        if a == 2:
+            db[b] = _f32_to_bf16_bits(_bf16_bits_to_f32(ob[b]) - xf)
+        elif a == 1:
+            ob[b] = _f32_to_bf16_bits(xf + _bf16_bits_to_f32(db[b]))
+    return ob, db
