@@ -143,6 +143,19 @@ int rapid3_gated_step_host(rapid3_ctx* ctx, const void* q_host, const void* k_ho
                            void* out_host, const int32_t* action_host, const float* keep_ratio_host, int B,
                            float softmax_scale, void* stream, int64_t* bytes_h2d, int64_t* bytes_d2h);
 
+/*
+ * Cache-Reuse data path (Sec. 3.2 "Level-2: Cache-Reuse", the conditional definition of O_t, and
+ * the cached residual Delta = G(X) - X).  x, o, delta: DEVICE bf16 arrays [B, elems_per_image],
+ * contiguous, 16-byte aligned; elems_per_image a multiple of 8.  Per image b:
+ *   action ATTEND: the generator has just written o[b]; the cache is refreshed, delta[b] = o[b] - x[b];
+ *   action REUSE : the cached residual replaces the generator,            o[b] = x[b] + delta[b];
+ *   action SKIP  : nothing is read or written.
+ * The sum / difference is taken in fp32 and rounded once to bf16.  Needs no context and no
+ * workspace; asynchronous on `stream`; if every image is skipped nothing is launched.
+ */
+int rapid3_cache_step(const void* x, void* o, void* delta, const int32_t* action_host, int B,
+                      int64_t elems_per_image, void* stream);
+
 /* Device pointers of the workspace rapid3_gated_step fills (any may be NULL): layouts as in
  * rapid3_block_scores / rapid3_select_mask with n_img = number of sparse images of the last step. */
 int rapid3_workspace(rapid3_ctx* ctx, float** scores, uint64_t** bitmask, int32_t** kept_idx,

@@ -22,7 +22,7 @@ EXPORTS = [
     "rapid3_create", "rapid3_destroy", "rapid3_strerror", "rapid3_num_blocks", "rapid3_mask_words",
     "rapid3_block_scores", "rapid3_select_mask", "rapid3_sparse_joint_attn", "rapid3_gated_step",
     "rapid3_gated_step_host", "rapid3_workspace", "rapid3_launch_count", "rapid3_last_status",
-    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes",
+    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step",
 ]
 
 
@@ -72,6 +72,7 @@ def load() -> ctypes.CDLL:
     lib.rapid3_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), i64p]
     lib.rapid3_block_scores_static.argtypes = [ctypes.POINTER(Shape), vp, vp, i32p, ci, vp, vp]
     lib.rapid3_static_scratch_bytes.argtypes = []
+    lib.rapid3_cache_step.argtypes = [vp, vp, vp, i32p, ci, ctypes.c_int64, vp]
     lib.rapid3_static_scratch_bytes.restype = ctypes.c_int64
     _lib = lib
     return lib
@@ -221,6 +222,15 @@ def rapid3_block_scores_static(shape: Shape, q: torch.Tensor, k: torch.Tensor, s
     _check(load().rapid3_block_scores_static(ctypes.byref(shape), _ptr(q), _ptr(k), _i32(img_idx), n, _ptr(scores),
                                              _stream()), "rapid3_block_scores_static")
     return scores
+
+
+def rapid3_cache_step(x: torch.Tensor, o: torch.Tensor, delta: torch.Tensor, actions: Sequence[int]):
+    """Cache-Reuse data path over a batch [B, ...] of contiguous bf16 tensors: refreshes `delta` for
+    attending images, writes `o` for reusing ones, leaves skipped ones alone."""
+    B = len(actions)
+    elems = x[0].numel()
+    _check(load().rapid3_cache_step(_ptr(x), _ptr(o), _ptr(delta), _i32(actions), B, elems, _stream()),
+           "rapid3_cache_step")
 
 
 def static_scratch_bytes() -> int:
