@@ -132,6 +132,21 @@ int rapid3_gated_step(rapid3_ctx* ctx, const void* q, const void* k, const void*
                       float softmax_scale, void* stream);
 
 /*
+ * The same step with the policy's decisions left on the GPU (Sec. 3.3: the heads sample their
+ * actions on the device; reading them back would cost a host synchronisation per step and layer):
+ * action_dev [B] int32 and keep_ratio_dev [B] float are DEVICE arrays, read by the kernels when
+ * they run on `stream`, not at call time.  A one-thread kernel builds the image lists, then the
+ * four kernels of rapid3_gated_step are launched with grids sized for all B images; thread blocks
+ * of images that do not attend return at once.  Results (output, workspace contents) are those of
+ * rapid3_gated_step with the same actions.  An action outside {SKIP, REUSE, ATTEND} or a ratio
+ * outside (0, 1] cannot be rejected at call time: that image is not processed and the device status
+ * word is set to RAPID3_ERR_INVALID_ARG (see rapid3_last_status).
+ */
+int rapid3_gated_step_device(rapid3_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                             const int32_t* action_dev, const float* keep_ratio_dev, int B,
+                             float softmax_scale, void* stream);
+
+/*
  * The same step with HOST tensors (pinned memory recommended): copies Q, K, V of the attending
  * images to device staging buffers, runs rapid3_gated_step and copies their rows of `out` back,
  * all on `stream`; gated images move no bytes.  The staging buffers (4 tensors of

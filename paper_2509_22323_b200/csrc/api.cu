@@ -38,6 +38,7 @@ struct rapid3_ctx {
     int32_t* kept_idx = nullptr;  // [B_max][H][nb][nb]
     int32_t* kept_cnt = nullptr;  // [B_max][H][nb]
     int* status = nullptr;
+    DevPlan* plan = nullptr;      // device-resident plan of rapid3_gated_step_device
     // host-tensor staging of rapid3_gated_step_host (created on first use)
     void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
     EncodeTiledFn encode = nullptr;
@@ -135,7 +136,7 @@ int get_map(rapid3_ctx* c, const void* base, const CUtensorMap** out) {
 
 int attn_launch(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out, const ImgList& l,
                 const int32_t* kept_idx, const int32_t* kept_cnt, const uint64_t* bitmask, float scale,
-                cudaStream_t st) {
+                cudaStream_t st, const DevPlan* plan = nullptr, int n_cap = 0) {
     const CUtensorMap *mq, *mk, *mv, *mo;
     int r;
     if ((r = get_map(c, q, &mq)) || (r = get_map(c, k, &mk)) || (r = get_map(c, v, &mv)) || (r = get_map(c, out, &mo)))
@@ -143,7 +144,7 @@ int attn_launch(rapid3_ctx* c, const void* q, const void* k, const void* v, void
     CUtensorMap tq = *mq, tk = *mk, tv = *mv, to = *mo;   // copies: a later get_map may recycle the slot
     {
         ProfScope ps(c, PROF_ATTN, st);
-        if (launch_attention(tq, tk, tv, to, c->g, l, kept_idx, kept_cnt, bitmask, scale, c->status, st) != cudaSuccess)
+        if (launch_attention(tq, tk, tv, to, c->g, l, kept_idx, kept_cnt, bitmask, scale, c->status, st, plan, n_cap) != cudaSuccess)
             return RAPID3_ERR_CUDA;
     }
     c->launches += 1;
@@ -214,7 +215,9 @@ int rapid3_create(rapid3_ctx** out, const rapid3_shape* shape) {
               cudaMalloc(&c->kept_idx, B * H * nb * nb * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&c->kept_cnt, B * H * nb * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&c->status, sizeof(int)) == cudaSuccess &&
-              cudaMemset(c->status, 0, sizeof(int)) == cudaSuccess;
+              cudaMemset(c->status, 0, sizeof(int)) == cudaSuccess &&
+              cudaMalloc(&c->plan, sizeof(DevPlan)) == cudaSuccess &&
+              cudaMemset(c->plan, 0, sizeof(DevPlan)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         rapid3_destroy(c);
@@ -237,6 +240,7 @@ int rapid3_destroy(rapid3_ctx* c) {
     cudaFree(c->kept_idx);
     cudaFree(c->kept_cnt);
     cudaFree(c->status);
+    cudaFree(c->plan);
     for (void* s : c->stage) cudaFree(s);
     for (auto& r : c->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     delete c;
@@ -359,6 +363,37 @@ int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v
     }
     return attn_launch(c, q, k, v, out, all, sparse.n ? c->kept_idx : nullptr, sparse.n ? c->kept_cnt : nullptr,
                        sparse.n ? c->bitmask : nullptr, softmax_scale, st);
+}
+
+int rapid3_gated_step_device(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
+                             const int32_t* action_dev, const float* keep_ratio_dev, int B, float softmax_scale,
+                             void* stream) {
+    if (!c || !q || !k || !v || !out || !action_dev || !keep_ratio_dev) return RAPID3_ERR_INVALID_ARG;
+    if (B < 1 || B > c->shape.B_max) return RAPID3_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return RAPID3_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q) % 16) || (reinterpret_cast<uintptr_t>(k) % 16)) return RAPID3_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The host never sees the actions: a one-thread kernel does the gate and compaction into the
+    // context's device-resident plan, and every following kernel is launched with a grid that covers
+    // all B images and takes its image list from the plan; the surplus CTAs return at once.
+    if (launch_plan(action_dev, keep_ratio_dev, B, c->g, c->plan, c->status, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+    ImgList none;
+    none.n = 0;
+    {
+        ProfScope ps(c, PROF_POOL, st);
+        if (launch_block_pool(q, k, c->g, none, c->pooled, st, c->plan, B) != cudaSuccess) return RAPID3_ERR_CUDA;
+    }
+    {
+        ProfScope ps(c, PROF_SCORES, st);
+        if (launch_block_scores(c->pooled, c->g, B, c->scores, st, c->plan) != cudaSuccess) return RAPID3_ERR_CUDA;
+    }
+    {
+        ProfScope ps(c, PROF_SELECT, st);
+        if (launch_select_mask(c->scores, c->g, none, c->bitmask, c->kept_idx, c->kept_cnt, st, c->plan, B) != cudaSuccess)
+            return RAPID3_ERR_CUDA;
+    }
+    c->launches += 4;
+    return attn_launch(c, q, k, v, out, none, c->kept_idx, c->kept_cnt, c->bitmask, softmax_scale, st, c->plan, B);
 }
 
 int rapid3_gated_step_host(rapid3_ctx* c, const void* q_host, const void* k_host, const void* v_host, void* out_host,

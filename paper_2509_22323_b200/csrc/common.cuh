@@ -22,6 +22,14 @@ struct ImgList {
     int k_free[RAPID3_MAX_IMG];
 };
 
+// Device-resident plan of one gated step (filled by plan_kernel from device-resident actions):
+// the two image lists the host path passes as kernel arguments.
+struct DevPlan {
+    ImgList sparse;   // images with keep ratio < 1, ascending batch order, slot = position
+    ImgList all;      // every attending image, descending keep ratio (dense first)
+    int n_dense;
+};
+
 struct TensorGeom {
     int H, D, N, nb, n_text_blocks;
     int pair_stride;                          // 1 or 2: which query blocks share an attention tile
@@ -29,17 +37,23 @@ struct TensorGeom {
 };
 
 // K1: block means of Q and K (fp64) for the listed images, then S = Qbar . Kbar^T -> fp32.
+// With `plan` set the image list is read from device memory (plan->sparse) and the grid is sized
+// for `n_cap` images; CTAs beyond the planned count return at once.  pooled is [2][n_cap][H][nb][D].
 cudaError_t launch_block_pool(const void* q, const void* k, const TensorGeom& g, const ImgList& imgs,
-                              double* pooled /* [2][n][H][nb][D] */, cudaStream_t s);
+                              double* pooled, cudaStream_t s, const DevPlan* plan = nullptr, int n_cap = 0);
 cudaError_t launch_block_scores(const double* pooled, const TensorGeom& g, int n_img, float* scores,
-                                cudaStream_t s);
+                                cudaStream_t s, const DevPlan* plan = nullptr);
 // K2: forced + top-k selection.
 cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const ImgList& imgs,
-                               uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s);
+                               uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s,
+                               const DevPlan* plan = nullptr, int n_cap = 0);
+// Builds the plan from device-resident actions and keep ratios (one thread; B <= RAPID3_MAX_IMG).
+cudaError_t launch_plan(const int32_t* action_dev, const float* ratio_dev, int B, const TensorGeom& g,
+                        DevPlan* plan, int* status, cudaStream_t s);
 // K3: attention over kept tiles.  `bitmask` (optional) is the select kernel's bitmask of the same
 // lists; when present the kernel reads it instead of walking the lists.
 cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv,
                              const CUtensorMap& tmo, const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
                              const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* status,
-                             cudaStream_t s);
+                             cudaStream_t s, const DevPlan* plan = nullptr, int n_cap = 0);
 cudaError_t attention_static_init();

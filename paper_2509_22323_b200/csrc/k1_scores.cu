@@ -16,16 +16,19 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 // same channels are then added with shuffles.  No shared memory.
 template <int D>
 __global__ void __launch_bounds__(128) pool_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k,
-                                                   TensorGeom g, ImgList imgs, double* __restrict__ pooled) {
+                                                   TensorGeom g, ImgList imgs, double* __restrict__ pooled,
+                                                   const DevPlan* __restrict__ plan, int n_cap) {
     constexpr int TPR = D / 8;          // lanes per token row (8 channels = 16 bytes each)
     constexpr int RPL = 32 / TPR;       // rows per warp-wide load
     constexpr int ITERS = 64 / RPL;     // loads per lane
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int blk = blockIdx.x * 4 + warp, h = blockIdx.y;
     if (blk >= g.nb) return;
-    const int which = blockIdx.z / imgs.n;            // 0 = Q, 1 = K
-    const int p = blockIdx.z - which * imgs.n;
-    const uint16_t* base = (which ? k : q) + (long long)imgs.batch[p] * g.stride_b + (long long)h * g.stride_h;
+    const int which = blockIdx.z / n_cap;             // 0 = Q, 1 = K
+    const int p = blockIdx.z - which * n_cap;
+    if (plan && p >= plan->sparse.n) return;          // device-resident plan: fewer images than the grid covers
+    const int batch = plan ? plan->sparse.batch[p] : imgs.batch[p];
+    const uint16_t* base = (which ? k : q) + (long long)batch * g.stride_b + (long long)h * g.stride_h;
     const int c = lane % TPR, r0 = lane / TPR;
     const int n0 = blk * 64;
     const int valid = min(64, g.N - n0);
@@ -56,7 +59,7 @@ __global__ void __launch_bounds__(128) pool_kernel(const uint16_t* __restrict__ 
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], off);
     if (lane < TPR) {
-        double* o = pooled + ((((long long)which * imgs.n + p) * g.H + h) * g.nb + blk) * D + c * 8;
+        double* o = pooled + ((((long long)which * n_cap + p) * g.H + h) * g.nb + blk) * D + c * 8;
         const double inv = 1.0 / (double)valid;
 #pragma unroll
         for (int e = 0; e < 8; e += 2) {
@@ -68,10 +71,11 @@ __global__ void __launch_bounds__(128) pool_kernel(const uint16_t* __restrict__ 
 
 // 32 x 32 tile of S per CTA, 16 x 16 threads, 2 x 2 outputs per thread, D in chunks of 32.
 __global__ void __launch_bounds__(256) scores_kernel(const double* __restrict__ pooled, TensorGeom g, int n_img,
-                                                     float* __restrict__ scores) {
+                                                     float* __restrict__ scores, const DevPlan* __restrict__ plan) {
     __shared__ double sq[32][33];
     __shared__ double sk[32][33];
     const int ph = blockIdx.z;                       // p * H + h
+    if (plan && ph >= plan->sparse.n * g.H) return;
     const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
     const double* pq = pooled + (long long)ph * g.nb * g.D;
     const double* pk = pooled + ((long long)n_img * g.H + ph) * g.nb * g.D;
@@ -102,19 +106,20 @@ __global__ void __launch_bounds__(256) scores_kernel(const double* __restrict__ 
 }  // namespace
 
 cudaError_t launch_block_pool(const void* q, const void* k, const TensorGeom& g, const ImgList& imgs,
-                              double* pooled, cudaStream_t s) {
-    dim3 grid((g.nb + 3) / 4, g.H, 2 * imgs.n);
+                              double* pooled, cudaStream_t s, const DevPlan* plan, int n_cap) {
+    if (!plan) n_cap = imgs.n;
+    dim3 grid((g.nb + 3) / 4, g.H, 2 * n_cap);
     if (g.D == 128)
-        pool_kernel<128><<<grid, 128, 0, s>>>((const uint16_t*)q, (const uint16_t*)k, g, imgs, pooled);
+        pool_kernel<128><<<grid, 128, 0, s>>>((const uint16_t*)q, (const uint16_t*)k, g, imgs, pooled, plan, n_cap);
     else
-        pool_kernel<64><<<grid, 128, 0, s>>>((const uint16_t*)q, (const uint16_t*)k, g, imgs, pooled);
+        pool_kernel<64><<<grid, 128, 0, s>>>((const uint16_t*)q, (const uint16_t*)k, g, imgs, pooled, plan, n_cap);
     return cudaGetLastError();
 }
 
 cudaError_t launch_block_scores(const double* pooled, const TensorGeom& g, int n_img, float* scores,
-                                cudaStream_t s) {
-    dim3 grid((g.nb + 31) / 32, (g.nb + 31) / 32, n_img * g.H);
-    scores_kernel<<<grid, 256, 0, s>>>(pooled, g, n_img, scores);
+                                cudaStream_t s, const DevPlan* plan) {
+    dim3 grid((g.nb + 31) / 32, (g.nb + 31) / 32, n_img * g.H);      // with a plan n_img is the capacity
+    scores_kernel<<<grid, 256, 0, s>>>(pooled, g, n_img, scores, plan);
     return cudaGetLastError();
 }
 

@@ -16,17 +16,18 @@ constexpr int WARPS = 4;
 __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restrict__ scores, TensorGeom g,
                                                             ImgList imgs, uint32_t* __restrict__ bitmask32,
                                                             int32_t* __restrict__ kept_idx,
-                                                            int32_t* __restrict__ kept_cnt, int words32) {
+                                                            int32_t* __restrict__ kept_cnt, int words32,
+                                                            const DevPlan* __restrict__ plan) {
     extern __shared__ float srow[];                       // [WARPS][nb_pad]
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int nb = g.nb, ntb = g.n_text_blocks;
     const int nb_pad = (nb + 31) & ~31;
     const long long row = (long long)blockIdx.x * WARPS + warp;        // (p * H + h) * nb + i
-    const long long n_rows = (long long)imgs.n * g.H * nb;
+    const long long n_rows = (long long)(plan ? plan->sparse.n : imgs.n) * g.H * nb;
     if (row >= n_rows) return;
     const int i = (int)(row % nb);
     const int p = (int)(row / ((long long)nb * g.H));
-    const int k = imgs.k_free[p];
+    const int k = plan ? plan->sparse.k_free[p] : imgs.k_free[p];
     uint32_t* s = reinterpret_cast<uint32_t*>(srow) + warp * nb_pad;
     const float* src = scores + row * nb;
     const bool text_row = i < ntb;
@@ -100,13 +101,75 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
 }  // namespace
 
 cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const ImgList& imgs, uint64_t* bitmask,
-                               int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s) {
-    const long long n_rows = (long long)imgs.n * g.H * g.nb;
+                               int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s, const DevPlan* plan, int n_cap) {
+    const long long n_rows = (long long)(plan ? n_cap : imgs.n) * g.H * g.nb;
     const int nb_pad = (g.nb + 31) & ~31;
     const int words32 = 2 * ((g.nb + 63) / 64);
     const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
     const size_t smem = (size_t)WARPS * nb_pad * sizeof(float);
     select_kernel<<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
-                                                 kept_cnt, words32);
+                                                 kept_cnt, words32, plan);
+    return cudaGetLastError();
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// Plan of a gated step from device-resident policy actions: the gate and compaction the host
+// entry point does on the CPU, for callers whose sampled actions never leave the GPU.
+namespace {
+
+__global__ void plan_kernel(const int32_t* __restrict__ action, const float* __restrict__ ratio, int B, int n_free_img,
+                            DevPlan* __restrict__ plan, int* __restrict__ status) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    ImgList& sp = plan->sparse;
+    ImgList& al = plan->all;
+    sp.n = 0;
+    al.n = 0;
+    int n_dense = 0;
+    float ratio_of[RAPID3_MAX_IMG];
+    for (int b = 0; b < B; ++b) {
+        const int a = action[b];
+        if (a != RAPID3_ACT_SKIP && a != RAPID3_ACT_REUSE && a != RAPID3_ACT_ATTEND) {
+            atomicExch(status, RAPID3_ERR_INVALID_ARG);       // unknown action: treated as a skip
+            continue;
+        }
+        if (a != RAPID3_ACT_ATTEND) continue;
+        const float r = ratio[b];
+        if (!(r > 0.f) || !(r <= 1.f)) {
+            atomicExch(status, RAPID3_ERR_INVALID_ARG);       // ratio outside (0, 1]: image not processed
+            continue;
+        }
+        int slot = -1;
+        if (r < 1.f) {
+            slot = sp.n++;
+            sp.batch[slot] = b;
+            sp.slot[slot] = slot;
+            double x = ceil((double)r * (double)n_free_img - 1e-6);
+            x = x < 0.0 ? 0.0 : (x > (double)n_free_img ? (double)n_free_img : x);
+            sp.k_free[slot] = (int)x;
+        } else {
+            ++n_dense;
+        }
+        int pos = al.n++;
+        while (pos > 0 && ratio_of[pos - 1] < r) {            // insertion sort, descending ratio, stable
+            al.batch[pos] = al.batch[pos - 1];
+            al.slot[pos] = al.slot[pos - 1];
+            ratio_of[pos] = ratio_of[pos - 1];
+            --pos;
+        }
+        al.batch[pos] = b;
+        al.slot[pos] = slot;
+        al.k_free[pos] = 0;
+        ratio_of[pos] = r;
+    }
+    plan->n_dense = n_dense;
+}
+
+}  // namespace
+
+cudaError_t launch_plan(const int32_t* action_dev, const float* ratio_dev, int B, const TensorGeom& g, DevPlan* plan,
+                        int* status, cudaStream_t s) {
+    const int n_free_img = g.nb - g.n_text_blocks - 1;
+    plan_kernel<<<1, 32, 0, s>>>(action_dev, ratio_dev, B, n_free_img > 0 ? n_free_img : 0, plan, status);
     return cudaGetLastError();
 }

@@ -47,6 +47,7 @@ struct AttnParams {
     const uint32_t* bitmask32;     // optional: the same mask as 32-bit words, [slot][H][nb][words32]
     int words32;
     int n_dense;                   // leading images of the list that keep every block
+    const DevPlan* plan;           // optional: image list and n_dense from device memory (grid sized for n_cap images)
     int* status;
     float scale_log2;
 };
@@ -107,11 +108,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     // longest-processing-time-first scheduling): every quad of the dense images and the quads of
     // the sparse images that hold a text query block walk all nb key blocks; the other quads of the
     // sparse images follow, image by image in the list's order (descending keep ratio).
-    int quad, h, p;
+    int quad, h, p, b, slot;
     {
         const int nq = (nb + 3) >> 2, ntq = min(nq, (g.n_text_blocks + 3) >> 2);
-        const int nd = prm.n_dense, ns = prm.imgs.n - nd;
+        const int n_all = prm.plan ? prm.plan->all.n : prm.imgs.n;
+        const int nd = prm.plan ? prm.plan->n_dense : prm.n_dense, ns = n_all - nd;
         int L = blockIdx.x;
+        if (L >= nq * g.H * n_all) return;               // device-resident plan: fewer images than the grid covers
         const int heavy_dense = nd * g.H * nq, heavy_sparse = ns * g.H * ntq;
         if (L < heavy_dense) {
             p = L / (g.H * nq); L -= p * g.H * nq;
@@ -126,8 +129,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             p = L / (g.H * nl); L -= p * g.H * nl; p += nd;
             h = L / nl; quad = ntq + (L - h * nl);
         }
+        b = prm.plan ? prm.plan->all.batch[p] : prm.imgs.batch[p];
+        slot = prm.plan ? prm.plan->all.slot[p] : prm.imgs.slot[p];
     }
-    const int b = prm.imgs.batch[p], slot = prm.imgs.slot[p];
     const int i0 = 4 * quad;
     // Which two of the quad's four query blocks form a 128-row tile: neighbours (a, a + 1), or, when
     // a row of the image grid spans two blocks, vertical neighbours (a, a + 2), whose kept lists
@@ -566,7 +570,7 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
                              const CUtensorMap& tmo,
                              const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
                              const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* status,
-                             cudaStream_t s) {
+                             cudaStream_t s, const DevPlan* plan, int n_cap) {
     if (!g_attr_set) {
         cudaError_t e = attention_static_init();
         if (e != cudaSuccess) return e;
@@ -583,7 +587,8 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
     int n_dense = 0;
     while (n_dense < imgs.n && (imgs.slot[n_dense] < 0 || kept_idx == nullptr)) ++n_dense;
     prm.n_dense = n_dense;
-    dim3 grid(((g.nb + 3) / 4) * g.H * imgs.n, 1, 1);
+    prm.plan = plan;
+    dim3 grid(((g.nb + 3) / 4) * g.H * (plan ? n_cap : imgs.n), 1, 1);
     if (g.D == 128)
         attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, tmo, prm);
     else
