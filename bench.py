@@ -356,6 +356,36 @@ def run_ours(args, wl):
         kernels["block_pool"]["achieved_gbs"] = pool_bytes / (pool_ms / pool_n * 1e-3) / 1e9
         kernels["block_pool"]["frac_of_hbm_peak"] = kernels["block_pool"]["achieved_gbs"] / peaks["hbm_gbs"]
 
+    # time of the same attention kernel at one keep ratio for the whole batch: ratio 1.0 is the dense
+    # reference, the others show how the time follows the kept-tile fraction
+    sweep = None
+    if not args.no_sweep and wl.steps == 1:
+        sweep = []
+        (Q, K, V) = sets[0]
+        for r in (1.0, 0.5, 0.25):
+            acts, ratios = [binding.ACT_ATTEND] * wl.batch, [r] * wl.batch
+            for _ in range(3):
+                ctx.rapid3_gated_step(Q, K, V, out, acts, ratios, wl.softmax_scale)
+            torch.cuda.synchronize()
+            if r < 1.0:
+                dm = binding.bitmask_to_dense(ctx.workspace(wl.batch, device=dev)[1], wl.n_blocks).numpy()
+                frac = float(dm.mean())
+            else:
+                frac = 1.0
+            ctx.profile(True)
+            ctx.profile_read()
+            for _ in range(20):
+                ctx.rapid3_gated_step(Q, K, V, out, acts, ratios, wl.softmax_scale)
+            torch.cuda.synchronize()
+            pr = ctx.profile_read()
+            ctx.profile(False)
+            step_ms = sum(v[0] for v in pr.values()) / 20.0
+            sweep.append({"keep_ratio": r, "kept_tile_fraction": frac, "attention_ms": pr["attention"][0] / pr["attention"][1],
+                          "all_kernels_ms": step_ms})
+        for e in sweep:
+            e["attention_speedup_vs_ratio_1"] = sweep[0]["attention_ms"] / e["attention_ms"]
+            e["step_speedup_vs_ratio_1"] = sweep[0]["all_kernels_ms"] / e["all_kernels_ms"]
+
     cpu = None
     if not args.no_cpu_baseline:
         v, secs, cores, desc = OracleSample(wl).run(args.cpu_budget)
@@ -371,7 +401,7 @@ def run_ours(args, wl):
                        "l2": f"inputs larger than L2 ({3 * sets[0][0].numel() * 2 / 1e6:.0f} MB per set), "
                              f"{nsets} input sets rotated"},
             "clocks": sampler.summary(w0, w1), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-            "cpu_baseline": cpu, "kernels": kernels}
+            "cpu_baseline": cpu, "kernels": kernels, "keep_ratio_sweep": sweep}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -386,6 +416,7 @@ def main():
     ap.add_argument("--workload", default="flux_1024", choices=list(inputs.WORKLOADS))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     if args.warmup < 3:
