@@ -156,7 +156,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         }
         for (int s = 0; s < 4; ++s) {
             mbar_init(bSF + 8 * s, 1);
-            mbar_init(bPF + 8 * s, 128);
+            mbar_init(bPF + 8 * s, 4);      // one arrival per softmax warp of the tile
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(bPV + 8 * t, 1);
@@ -484,7 +484,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             }
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(bPFt + 8 * buf);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bPFt + 8 * buf);
             ++n;
         }
         // epilogue: O / l -> bf16 -> the tile's (now unused) Q buffer in the 128-byte swizzled layout
