@@ -41,6 +41,9 @@ struct rapid3_ctx {
     DevPlan* plan = nullptr;      // device-resident plan of rapid3_gated_step_device
     // host-tensor staging of rapid3_gated_step_host (created on first use)
     void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
+    cudaStream_t up_s = nullptr, down_s = nullptr;            // copy streams of the host entry
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    std::vector<cudaEvent_t> ev_up, ev_done;                  // per image: inputs landed / output computed
     EncodeTiledFn encode = nullptr;
     MapSlot maps[6];              // small cache keyed by base pointer
     int map_rr = 0;
@@ -242,6 +245,12 @@ int rapid3_destroy(rapid3_ctx* c) {
     cudaFree(c->status);
     cudaFree(c->plan);
     for (void* s : c->stage) cudaFree(s);
+    if (c->up_s) cudaStreamDestroy(c->up_s);
+    if (c->down_s) cudaStreamDestroy(c->down_s);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    for (cudaEvent_t e : c->ev_up) cudaEventDestroy(e);
+    for (cudaEvent_t e : c->ev_done) cudaEventDestroy(e);
     for (auto& r : c->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     delete c;
     return RAPID3_OK;
@@ -408,36 +417,72 @@ int rapid3_gated_step_host(rapid3_ctx* c, const void* q_host, const void* k_host
     if (s.stride_n != s.D || s.stride_h != N * s.D || s.stride_b != (long long)s.H * N * s.D)
         return RAPID3_ERR_UNSUPPORTED;
     const size_t img_bytes = (size_t)s.H * N * s.D * 2;
+    for (int b = 0; b < B; ++b) {
+        const int a = action_host[b];
+        if (a != RAPID3_ACT_SKIP && a != RAPID3_ACT_REUSE && a != RAPID3_ACT_ATTEND) return RAPID3_ERR_INVALID_ARG;
+        if (a == RAPID3_ACT_ATTEND && (!(keep_ratio_host[b] > 0.f) || !(keep_ratio_host[b] <= 1.f)))
+            return RAPID3_ERR_INVALID_ARG;
+    }
+    if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return RAPID3_ERR_INVALID_ARG;
     if (!c->stage[0]) {
-        for (int i = 0; i < 4; ++i)
-            if (cudaMalloc(&c->stage[i], img_bytes * s.B_max) != cudaSuccess) {
-                cudaGetLastError();
-                for (int j = 0; j < 4; ++j) { cudaFree(c->stage[j]); c->stage[j] = nullptr; }
-                return RAPID3_ERR_WORKSPACE;
-            }
+        bool ok = true;
+        for (int i = 0; i < 4 && ok; ++i) ok = cudaMalloc(&c->stage[i], img_bytes * s.B_max) == cudaSuccess;
+        ok = ok && cudaStreamCreateWithFlags(&c->up_s, cudaStreamNonBlocking) == cudaSuccess &&
+             cudaStreamCreateWithFlags(&c->down_s, cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
+        for (int b = 0; b < s.B_max && ok; ++b) {
+            cudaEvent_t e0 = nullptr, e1 = nullptr;
+            ok = cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) == cudaSuccess;
+            if (e0) c->ev_up.push_back(e0);
+            if (e1) c->ev_done.push_back(e1);
+        }
+        if (!ok) {
+            cudaGetLastError();
+            for (int j = 0; j < 4; ++j) { cudaFree(c->stage[j]); c->stage[j] = nullptr; }
+            return RAPID3_ERR_WORKSPACE;
+        }
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const void* src[3] = {q_host, k_host, v_host};
     int64_t up = 0, down = 0;
+    // Image by image: inputs go up on one copy stream, the step of that image runs on `stream` as soon
+    // as they have landed, its output goes down on a second copy stream -- so the uploads of the next
+    // images, the compute and the downloads overlap (the link is full duplex).  Everything is forked
+    // from and joined back into `stream`.
+    if (cudaEventRecord(c->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(c->up_s, c->ev_fork, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(c->down_s, c->ev_fork, 0) != cudaSuccess)
+        return RAPID3_ERR_CUDA;
+    int32_t one[RAPID3_MAX_IMG];
+    for (int b = 0; b < B; ++b) one[b] = RAPID3_ACT_SKIP;
+    bool any = false;
     for (int b = 0; b < B; ++b) {
         if (action_host[b] != RAPID3_ACT_ATTEND) continue;
+        any = true;
         for (int i = 0; i < 3; ++i) {
             if (cudaMemcpyAsync((char*)c->stage[i] + b * img_bytes, (const char*)src[i] + b * img_bytes, img_bytes,
-                                cudaMemcpyHostToDevice, st) != cudaSuccess)
+                                cudaMemcpyHostToDevice, c->up_s) != cudaSuccess)
                 return RAPID3_ERR_CUDA;
             up += (int64_t)img_bytes;
         }
-    }
-    int r = rapid3_gated_step(c, c->stage[0], c->stage[1], c->stage[2], c->stage[3], action_host, keep_ratio_host, B,
-                              softmax_scale, stream);
-    if (r != RAPID3_OK) return r;
-    for (int b = 0; b < B; ++b) {
-        if (action_host[b] != RAPID3_ACT_ATTEND) continue;
+        if (cudaEventRecord(c->ev_up[b], c->up_s) != cudaSuccess || cudaStreamWaitEvent(st, c->ev_up[b], 0) != cudaSuccess)
+            return RAPID3_ERR_CUDA;
+        one[b] = RAPID3_ACT_ATTEND;
+        const int r = rapid3_gated_step(c, c->stage[0], c->stage[1], c->stage[2], c->stage[3], one, keep_ratio_host, B,
+                                        softmax_scale, stream);
+        one[b] = RAPID3_ACT_SKIP;
+        if (r != RAPID3_OK) return r;
+        if (cudaEventRecord(c->ev_done[b], st) != cudaSuccess ||
+            cudaStreamWaitEvent(c->down_s, c->ev_done[b], 0) != cudaSuccess)
+            return RAPID3_ERR_CUDA;
         if (cudaMemcpyAsync((char*)out_host + b * img_bytes, (const char*)c->stage[3] + b * img_bytes, img_bytes,
-                            cudaMemcpyDeviceToHost, st) != cudaSuccess)
+                            cudaMemcpyDeviceToHost, c->down_s) != cudaSuccess)
             return RAPID3_ERR_CUDA;
         down += (int64_t)img_bytes;
     }
+    if (any && (cudaEventRecord(c->ev_join, c->down_s) != cudaSuccess || cudaStreamWaitEvent(st, c->ev_join, 0) != cudaSuccess))
+        return RAPID3_ERR_CUDA;
     if (bytes_h2d) *bytes_h2d = up;
     if (bytes_d2h) *bytes_d2h = down;
     return RAPID3_OK;
