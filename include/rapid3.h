@@ -132,6 +132,21 @@ int rapid3_gated_step(rapid3_ctx* ctx, const void* q, const void* k, const void*
                       float softmax_scale, void* stream);
 
 /*
+ * The same step with one keep ratio per (image, head): keep_ratio_host is [B][H], row-major
+ * (Sec. 3.2: the sparsity head emits a ratio for every layer and head).  Head h of image b keeps
+ * clamp(ceil(keep_ratio_host[b][h] * n_free - 1e-6)) free candidates per query-block row; forced
+ * blocks are as in rapid3_select_mask.  An image whose H ratios are all exactly 1 is dense and
+ * skips scoring and selection; any other attending image is scored once and selected per head.
+ * Every ratio of an attending image must lie in (0, 1], else RAPID3_ERR_INVALID_ARG; the ratios of
+ * gated images are ignored.  The keep counts travel as a kernel argument, so (sparse images) * H
+ * may not exceed 2048: more returns RAPID3_ERR_UNSUPPORTED and launches nothing.  Workspace
+ * layout and everything else are as in rapid3_gated_step.
+ */
+int rapid3_gated_step_heads(rapid3_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                            const int32_t* action_host, const float* keep_ratio_host, int B,
+                            float softmax_scale, void* stream);
+
+/*
  * The same step with the policy's decisions left on the GPU (Sec. 3.3: the heads sample their
  * actions on the device; reading them back would cost a host synchronisation per step and layer):
  * action_dev [B] int32 and keep_ratio_dev [B] float are DEVICE arrays, read by the kernels when

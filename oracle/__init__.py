@@ -180,6 +180,15 @@ def image_mask(q, k, n_text: int, ratio: float):
     return S32, mask, gap
 
 
+def image_mask_heads(q, k, n_text: int, ratios: Sequence[float]):
+    """The same with one keep ratio per head (Sec. 3.2: the sparsity head emits theta in R^{L x H}):
+    head h is selected on its own scores with ratios[h]."""
+    S32 = image_scores(q, k)
+    assert len(ratios) == S32.shape[0]
+    parts = [select_mask(S32[h:h + 1].astype(np.float64), n_text, float(r)) for h, r in enumerate(ratios)]
+    return S32, np.concatenate([m for m, _ in parts]), np.concatenate([g for _, g in parts])
+
+
 def sparse_joint_attention(q, k, v, n_text: int, ratio: float, scale: float, qb_lo: int = 0,
                            qb_hi: Optional[int] = None, heads: Optional[Sequence[int]] = None):
     """Whole path for one image: returns dict(scores, mask, gap, out)."""

@@ -22,7 +22,7 @@ EXPORTS = [
     "rapid3_create", "rapid3_destroy", "rapid3_strerror", "rapid3_num_blocks", "rapid3_mask_words",
     "rapid3_block_scores", "rapid3_select_mask", "rapid3_sparse_joint_attn", "rapid3_gated_step",
     "rapid3_gated_step_host", "rapid3_workspace", "rapid3_launch_count", "rapid3_last_status",
-    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device",
+    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device", "rapid3_gated_step_heads",
 ]
 
 
@@ -63,6 +63,7 @@ def load() -> ctypes.CDLL:
     lib.rapid3_select_mask.argtypes = [vp, vp, f32p, ci, vp, vp, vp, vp]
     lib.rapid3_sparse_joint_attn.argtypes = [vp, vp, vp, vp, vp, i32p, ci, vp, vp, cf, vp]
     lib.rapid3_gated_step.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp]
+    lib.rapid3_gated_step_heads.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp]
     lib.rapid3_gated_step_device.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, cf, vp]
     lib.rapid3_gated_step_host.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp, i64p, i64p]
     lib.rapid3_workspace.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
@@ -171,6 +172,17 @@ class Context:
         scale = softmax_scale if softmax_scale is not None else self.D ** -0.5
         _check(self.lib.rapid3_gated_step(self.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _i32(actions),
                                           _f32(keep_ratio), len(actions), scale, _stream()), "rapid3_gated_step")
+        return out
+
+    def rapid3_gated_step_heads(self, q, k, v, out, actions: Sequence[int], keep_ratio: Sequence[Sequence[float]],
+                                softmax_scale: Optional[float] = None):
+        """keep_ratio: [B][H], one ratio per image and head."""
+        scale = softmax_scale if softmax_scale is not None else self.D ** -0.5
+        flat = [float(r) for row in keep_ratio for r in row]
+        assert len(flat) == len(actions) * self.H
+        _check(self.lib.rapid3_gated_step_heads(self.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _i32(actions),
+                                                _f32(flat), len(actions), scale, _stream()),
+               "rapid3_gated_step_heads")
         return out
 
     def rapid3_gated_step_device(self, q, k, v, out, actions_dev: torch.Tensor, keep_ratio_dev: torch.Tensor,

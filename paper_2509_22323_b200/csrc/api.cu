@@ -313,9 +313,11 @@ int rapid3_sparse_joint_attn(rapid3_ctx* c, const void* q, const void* k, const 
                        static_cast<cudaStream_t>(stream));
 }
 
-int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
-                      const int32_t* action_host, const float* keep_ratio_host, int B, float softmax_scale,
-                      void* stream) {
+// One gated step.  heads_per_ratio == 1: keep_ratio_host is [B].  heads_per_ratio == H: it is
+// [B][H], one ratio per (image, head); an image is dense only when all its heads keep everything.
+static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
+                           const int32_t* action_host, const float* keep_ratio_host, int heads_per_ratio, int B,
+                           float softmax_scale, void* stream) {
     if (!c || !q || !k || !v || !out || !action_host || !keep_ratio_host) return RAPID3_ERR_INVALID_ARG;
     if (B < 1 || B > c->shape.B_max) return RAPID3_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return RAPID3_ERR_INVALID_ARG;
@@ -327,11 +329,25 @@ int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v
     sparse.n = 0;
     all.n = 0;
     float ratio_of[RAPID3_MAX_IMG];
+    const bool per_head = heads_per_ratio > 1;
+    const int H = c->g.H;
+    HeadKeep hk;
     for (int b = 0; b < B; ++b) {
         const int a = action_host[b];
         if (a != RAPID3_ACT_SKIP && a != RAPID3_ACT_REUSE && a != RAPID3_ACT_ATTEND) return RAPID3_ERR_INVALID_ARG;
         if (a != RAPID3_ACT_ATTEND) continue;
-        const float ratio = keep_ratio_host[b];
+        float ratio = keep_ratio_host[(size_t)b * heads_per_ratio];
+        if (per_head) {                                   // order images by their mean ratio
+            double sum = 0.0;
+            bool all_one = true;
+            for (int h = 0; h < H; ++h) {
+                const float rh = keep_ratio_host[(size_t)b * H + h];
+                if (!(rh > 0.f) || !(rh <= 1.f)) return RAPID3_ERR_INVALID_ARG;
+                sum += rh;
+                all_one = all_one && rh == 1.f;
+            }
+            ratio = all_one ? 1.f : fminf((float)(sum / H), 0.99999994f);
+        }
         if (!(ratio > 0.f) || !(ratio <= 1.f)) return RAPID3_ERR_INVALID_ARG;
         int slot = -1;
         if (ratio < 1.f) {
@@ -339,6 +355,12 @@ int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v
             sparse.batch[slot] = b;
             sparse.slot[slot] = slot;
             sparse.k_free[slot] = keep_count((double)ratio, n_free_img > 0 ? n_free_img : 0);
+            if (per_head) {
+                if ((slot + 1) * H > RAPID3_MAX_HEAD_ROWS) return RAPID3_ERR_UNSUPPORTED;
+                for (int h = 0; h < H; ++h)
+                    hk.k[slot * H + h] =
+                        keep_count((double)keep_ratio_host[(size_t)b * H + h], n_free_img > 0 ? n_free_img : 0);
+            }
         }
         int pos = all.n++;
         while (pos > 0 && ratio_of[pos - 1] < ratio) {   // insertion sort, descending ratio, stable
@@ -365,13 +387,30 @@ int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v
         }
         {
             ProfScope ps(c, PROF_SELECT, st);
-            if (launch_select_mask(c->scores, c->g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st) != cudaSuccess)
-                return RAPID3_ERR_CUDA;
+            const cudaError_t e =
+                per_head ? launch_select_mask_heads(c->scores, c->g, sparse, hk, c->bitmask, c->kept_idx, c->kept_cnt, st)
+                         : launch_select_mask(c->scores, c->g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st);
+            if (e != cudaSuccess) return RAPID3_ERR_CUDA;
         }
         c->launches += 3;
     }
     return attn_launch(c, q, k, v, out, all, sparse.n ? c->kept_idx : nullptr, sparse.n ? c->kept_cnt : nullptr,
                        sparse.n ? c->bitmask : nullptr, softmax_scale, st);
+}
+
+int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
+                      const int32_t* action_host, const float* keep_ratio_host, int B, float softmax_scale,
+                      void* stream) {
+    return gated_step_impl(c, q, k, v, out, action_host, keep_ratio_host, 1, B, softmax_scale, stream);
+}
+
+int rapid3_gated_step_heads(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
+                            const int32_t* action_host, const float* keep_ratio_host, int B, float softmax_scale,
+                            void* stream) {
+    if (!c) return RAPID3_ERR_INVALID_ARG;
+    if (c->g.H == 1)
+        return gated_step_impl(c, q, k, v, out, action_host, keep_ratio_host, 1, B, softmax_scale, stream);
+    return gated_step_impl(c, q, k, v, out, action_host, keep_ratio_host, c->g.H, B, softmax_scale, stream);
 }
 
 int rapid3_gated_step_device(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,

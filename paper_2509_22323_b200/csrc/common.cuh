@@ -30,6 +30,17 @@ struct DevPlan {
     int n_dense;
 };
 
+// Keep counts per (sparse slot, head) for a policy that sets one ratio per head (Sec. 3.2: the
+// sparsity head emits theta in R^{L x H}).  Travels as a kernel argument, so slots * H is bounded.
+#define RAPID3_MAX_HEAD_ROWS 2048
+struct HeadKeep {
+    static constexpr bool per_head = true;
+    int k[RAPID3_MAX_HEAD_ROWS];
+};
+struct NoHeadKeep {
+    static constexpr bool per_head = false;
+};
+
 struct TensorGeom {
     int H, D, N, nb, n_text_blocks;
     int pair_stride;                          // 1 or 2: which query blocks share an attention tile
@@ -47,6 +58,9 @@ cudaError_t launch_block_scores(const double* pooled, const TensorGeom& g, int n
 cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const ImgList& imgs,
                                uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s,
                                const DevPlan* plan = nullptr, int n_cap = 0);
+cudaError_t launch_select_mask_heads(const float* scores, const TensorGeom& g, const ImgList& imgs,
+                                     const HeadKeep& hk, uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt,
+                                     cudaStream_t s);
 // Builds the plan from device-resident actions and keep ratios (one thread; B <= RAPID3_MAX_IMG).
 cudaError_t launch_plan(const int32_t* action_dev, const float* ratio_dev, int B, const TensorGeom& g,
                         DevPlan* plan, int* status, cudaStream_t s);

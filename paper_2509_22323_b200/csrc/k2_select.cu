@@ -13,11 +13,13 @@ namespace {
 
 constexpr int WARPS = 4;
 
+// HK = HeadKeep: one keep count per (image, head), passed by value.  HK = NoHeadKeep: per image.
+template <typename HK>
 __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restrict__ scores, TensorGeom g,
                                                             ImgList imgs, uint32_t* __restrict__ bitmask32,
                                                             int32_t* __restrict__ kept_idx,
                                                             int32_t* __restrict__ kept_cnt, int words32,
-                                                            const DevPlan* __restrict__ plan) {
+                                                            const DevPlan* __restrict__ plan, const HK hk) {
     extern __shared__ float srow[];                       // [WARPS][nb_pad]
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int nb = g.nb, ntb = g.n_text_blocks;
@@ -27,7 +29,11 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
     if (row >= n_rows) return;
     const int i = (int)(row % nb);
     const int p = (int)(row / ((long long)nb * g.H));
-    const int k = plan ? plan->sparse.k_free[p] : imgs.k_free[p];
+    // free candidates kept in this row: one count per image, or per (image, head) when the policy
+    // sets a ratio for every head
+    int k;
+    if constexpr (HK::per_head) k = hk.k[p * g.H + (int)((row / nb) % g.H)];
+    else k = plan ? plan->sparse.k_free[p] : imgs.k_free[p];
     uint32_t* s = reinterpret_cast<uint32_t*>(srow) + warp * nb_pad;
     const float* src = scores + row * nb;
     const bool text_row = i < ntb;
@@ -107,8 +113,20 @@ cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const I
     const int words32 = 2 * ((g.nb + 63) / 64);
     const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
     const size_t smem = (size_t)WARPS * nb_pad * sizeof(float);
-    select_kernel<<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
-                                                 kept_cnt, words32, plan);
+    select_kernel<NoHeadKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
+                                                        kept_cnt, words32, plan, NoHeadKeep());
+    return cudaGetLastError();
+}
+
+cudaError_t launch_select_mask_heads(const float* scores, const TensorGeom& g, const ImgList& imgs, const HeadKeep& hk,
+                                     uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s) {
+    const long long n_rows = (long long)imgs.n * g.H * g.nb;
+    const int nb_pad = (g.nb + 31) & ~31;
+    const int words32 = 2 * ((g.nb + 63) / 64);
+    const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
+    const size_t smem = (size_t)WARPS * nb_pad * sizeof(float);
+    select_kernel<HeadKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
+                                                       kept_cnt, words32, nullptr, hk);
     return cudaGetLastError();
 }
 

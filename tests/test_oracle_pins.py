@@ -121,6 +121,32 @@ def test_kept_count_identity_and_structure(nb, n_text):
     assert prev.all()                               # ratio 1.0 keeps everything
 
 
+def test_per_head_ratios_select_each_head_on_its_own():
+    # a head's mask depends on that head's scores and ratio alone: brute force per head, and the
+    # heads must not leak into each other (swapping two ratios swaps nothing but the counts)
+    rng = np.random.default_rng(5)
+    H, N, D, n_text = 3, 7 * 64 + 9, 16, 70
+    qt, kt, _ = rand_qkv(rng, H, N, D)
+    ratios = [0.2, 1.0, 0.6]
+    S32, mask, gap = oracle.image_mask_heads(qt, kt, n_text, ratios)
+    nb, ntb = 8, 2
+    assert mask.shape == (H, nb, nb) and gap.shape == (H, nb)
+    S = S32.astype(np.float64)
+    for h, r in enumerate(ratios):
+        for i in range(ntb, nb):
+            free = [j for j in range(ntb, nb) if j != i]
+            kk = oracle.keep_count(r, len(free))
+            best = max(itertools.combinations(free, kk), key=lambda c: sum(S[h, i, j] for j in c))
+            assert [j for j in free if mask[h, i, j]] == sorted(best)
+            assert mask[h, i, :ntb].all() and mask[h, i, i]
+        assert mask[h, :ntb].all()
+    assert mask[1].all()
+    # one ratio for all heads is the per-image rule
+    _, m_same, _ = oracle.image_mask_heads(qt, kt, n_text, [0.6] * H)
+    _, m_img, _ = oracle.image_mask(qt, kt, n_text, 0.6)
+    assert (m_same == m_img).all() and (m_same[2] == mask[2]).all()
+
+
 def test_keep_count_rounding():
     assert oracle.keep_count(0.5, 63) == 32
     assert oracle.keep_count(0.25, 63) == 16
