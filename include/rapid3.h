@@ -235,6 +235,20 @@ int rapid3_block_scores_static(const rapid3_shape* shape, const void* q, const v
 /* Size in bytes of the fixed scratch array of rapid3_block_scores_static. */
 int64_t rapid3_static_scratch_bytes(void);
 
+/*
+ * Cost report of one sampling trajectory (Sec. 3.3, "equivalent steps"): host arithmetic only.
+ *   K = sum over the steps that run of (1 - C_cache[k]) * (1 - C_sparse[k]),
+ * where C_cache[k] is the cost reduction of a step that reuses the cache and C_sparse[k] that of a
+ * step that attends sparsely, both in [0, 1].  action_host[k] says what step k did: a SKIP step
+ * does not run and adds nothing; a REUSE step adds 1 - c_cache_host[k] (it runs no attention, so
+ * no sparse reduction applies); an ATTEND step adds 1 - c_sparse_host[k] (0 for dense attention).
+ * *k_exact (may be NULL) receives the sum in fp64, *k_rounded (may be NULL) the nearest integer,
+ * halves upward.  n_steps >= 0.  A reduction outside [0, 1] or an unknown action returns
+ * RAPID3_ERR_INVALID_ARG and writes nothing.  No GPU work, no context.
+ */
+int rapid3_equivalent_steps(const int32_t* action_host, const float* c_cache_host, const float* c_sparse_host,
+                            int n_steps, double* k_exact, int64_t* k_rounded);
+
 /* Copies the device status word to *device_status (RAPID3_OK or a negative code) and clears it.
  * Synchronises the device; call it after the stream has been synchronised. */
 int rapid3_last_status(rapid3_ctx* ctx, int* device_status);

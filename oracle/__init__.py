@@ -237,3 +237,19 @@ def cache_step(x, o, delta, actions: Sequence[int]):
         elif a == 1:
             ob[b] = _f32_to_bf16_bits(xf + _bf16_bits_to_f32(db[b]))
     return ob, db
+
+
+# ----------------------------------------------------------------------------------------------
+# Equivalent steps (paper Sec. 3.3, the cost term of the reward): K = sum_k (1 - C_k^cache) *
+# (1 - C_k^sparse) over the steps the step policy keeps, rounded to the nearest integer.  A step
+# that reuses the cache has C^sparse = 0 (no attention runs), a step that attends has C^cache = 0.
+
+def equivalent_steps(actions: Sequence[int], c_cache: Sequence[float], c_sparse: Sequence[float]):
+    total = 0.0
+    for a, cc, cs in zip(actions, c_cache, c_sparse):
+        if a == 0:                      # skipped: the step is not part of the trajectory
+            continue
+        C_cache = float(np.float32(cc)) if a == 1 else 0.0
+        C_sparse = float(np.float32(cs)) if a == 2 else 0.0
+        total += (1.0 - C_cache) * (1.0 - C_sparse)
+    return total, int(np.floor(total + 0.5))

@@ -22,7 +22,7 @@ EXPORTS = [
     "rapid3_create", "rapid3_destroy", "rapid3_strerror", "rapid3_num_blocks", "rapid3_mask_words",
     "rapid3_block_scores", "rapid3_select_mask", "rapid3_sparse_joint_attn", "rapid3_gated_step",
     "rapid3_gated_step_host", "rapid3_workspace", "rapid3_launch_count", "rapid3_last_status",
-    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device", "rapid3_gated_step_heads",
+    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device", "rapid3_gated_step_heads", "rapid3_equivalent_steps",
 ]
 
 
@@ -74,6 +74,7 @@ def load() -> ctypes.CDLL:
     lib.rapid3_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), i64p]
     lib.rapid3_block_scores_static.argtypes = [ctypes.POINTER(Shape), vp, vp, i32p, ci, vp, vp]
     lib.rapid3_static_scratch_bytes.argtypes = []
+    lib.rapid3_equivalent_steps.argtypes = [i32p, f32p, f32p, ci, ctypes.POINTER(ctypes.c_double), i64p]
     lib.rapid3_cache_step.argtypes = [vp, vp, vp, i32p, ci, ctypes.c_int64, vp]
     lib.rapid3_static_scratch_bytes.restype = ctypes.c_int64
     _lib = lib
@@ -245,6 +246,16 @@ def rapid3_block_scores_static(shape: Shape, q: torch.Tensor, k: torch.Tensor, s
     _check(load().rapid3_block_scores_static(ctypes.byref(shape), _ptr(q), _ptr(k), _i32(img_idx), n, _ptr(scores),
                                              _stream()), "rapid3_block_scores_static")
     return scores
+
+
+def rapid3_equivalent_steps(actions: Sequence[int], c_cache: Sequence[float], c_sparse: Sequence[float]):
+    """Equivalent steps K of one trajectory: (exact sum, nearest integer)."""
+    n = len(actions)
+    assert len(c_cache) == n and len(c_sparse) == n
+    k, kr = ctypes.c_double(0.0), ctypes.c_int64(0)
+    _check(load().rapid3_equivalent_steps(_i32(actions), _f32(c_cache), _f32(c_sparse), n, ctypes.byref(k),
+                                          ctypes.byref(kr)), "rapid3_equivalent_steps")
+    return k.value, kr.value
 
 
 def rapid3_cache_step(x: torch.Tensor, o: torch.Tensor, delta: torch.Tensor, actions: Sequence[int]):

@@ -569,3 +569,19 @@ int rapid3_last_status(rapid3_ctx* c, int* device_status) {
 }
 
 }  // extern "C"
+
+int rapid3_equivalent_steps(const int32_t* action_host, const float* c_cache_host, const float* c_sparse_host,
+                            int n_steps, double* k_exact, int64_t* k_rounded) {
+    if (n_steps < 0 || (n_steps > 0 && (!action_host || !c_cache_host || !c_sparse_host))) return RAPID3_ERR_INVALID_ARG;
+    double sum = 0.0;
+    for (int s = 0; s < n_steps; ++s) {
+        const int a = action_host[s];
+        if (a == RAPID3_ACT_SKIP) continue;
+        const float c = a == RAPID3_ACT_REUSE ? c_cache_host[s] : c_sparse_host[s];
+        if ((a != RAPID3_ACT_REUSE && a != RAPID3_ACT_ATTEND) || !(c >= 0.f) || !(c <= 1.f)) return RAPID3_ERR_INVALID_ARG;
+        sum += 1.0 - (double)c;
+    }
+    if (k_exact) *k_exact = sum;
+    if (k_rounded) *k_rounded = (int64_t)floor(sum + 0.5);
+    return RAPID3_OK;
+}
