@@ -59,6 +59,7 @@ def _load():
         lib.oracle_keep_count.argtypes = [cd, ci]
         lib.oracle_keep_count.restype = ci
         lib.oracle_select_mask.argtypes = [f64p, ci, ci, cd, u8p, f64p]
+        lib.oracle_select_mask_mass.argtypes = [f64p, ci, ci, cd, cd, u8p, f64p, ctypes.POINTER(ctypes.c_int32), f64p]
         lib.oracle_masked_attention.argtypes = [u16p, u16p, u16p, ci, ci, u8p, cd, ci, ci, f64p]
         lib.oracle_attention_weights.argtypes = [u16p, u16p, ci, ci, u8p, cd, ci, f64p]
         lib.oracle_num_threads.restype = ci
@@ -135,6 +136,23 @@ def select_mask(S: np.ndarray, n_text: int, ratio: float):
     return mask, gap
 
 
+def select_mask_mass(S: np.ndarray, n_text: int, tau: float, scale: float):
+    """Cumulative-mass selection: [H, nb, nb] scores -> (mask uint8 [H, nb, nb], gap fp64 [H, nb],
+    k int32 [H, nb] free candidates kept per row, margin fp64 [H, nb])."""
+    S = np.ascontiguousarray(S, dtype=np.float64)
+    H, nb, _ = S.shape
+    mask = np.zeros((H, nb, nb), dtype=np.uint8)
+    gap = np.empty((H, nb), dtype=np.float64)
+    k = np.empty((H, nb), dtype=np.int32)
+    margin = np.empty((H, nb), dtype=np.float64)
+    lib = _load()
+    for h in range(H):
+        lib.oracle_select_mask_mass(_p(S[h], ctypes.c_double), nb, n_text_blocks(n_text), float(tau), float(scale),
+                                    _p(mask[h], ctypes.c_uint8), _p(gap[h], ctypes.c_double),
+                                    _p(k[h], ctypes.c_int32), _p(margin[h], ctypes.c_double))
+    return mask, gap, k, margin
+
+
 def masked_attention(q, k, v, mask: np.ndarray, scale: float, qb_lo: int = 0, qb_hi: Optional[int] = None,
                      heads: Optional[Sequence[int]] = None) -> np.ndarray:
     """[H, N, D] bf16 Q, K, V and mask [H, nb, nb] -> fp64 [H, N, D].
@@ -178,6 +196,14 @@ def image_mask(q, k, n_text: int, ratio: float):
     S32 = image_scores(q, k)
     mask, gap = select_mask(S32.astype(np.float64), n_text, ratio)
     return S32, mask, gap
+
+
+def image_mask_mass(q, k, n_text: int, tau: float, scale: float):
+    """Scores (fp32) and the cumulative-mass mask of one image; the weights are taken on the fp32
+    scores with the scale as an fp32 number, the arithmetic itself is fp64."""
+    S32 = image_scores(q, k)
+    mask, gap, kk, margin = select_mask_mass(S32.astype(np.float64), n_text, tau, float(np.float32(scale)))
+    return S32, mask, gap, kk, margin
 
 
 def image_mask_heads(q, k, n_text: int, ratios: Sequence[float]):

@@ -114,6 +114,72 @@ void oracle_select_mask(const double *S, int nb, int n_text_blocks, double ratio
     free(cand);
 }
 
+/* Cumulative-mass variant of steps 4-5 (Sec. 3.2: the sparse candidates are thresholds, not
+ * counts; the paper leaves the rule to the sparse-attention method it plugs in, so this is the
+ * plain "smallest set of the best blocks that holds a share tau of the row's mass" rule).
+ * Forced blocks as above.  For the free candidates of row i, in the order (score descending,
+ * index ascending):
+ *     w_c   = exp(scale * (S[i, c] - max over the free candidates of S[i, .]))
+ *     k     = the smallest count whose first k weights sum to at least tau * (sum of all w);
+ *             all of them when tau >= 1, none when there is no candidate
+ * and the first k candidates are kept.
+ * k_out[i]  = k (0 for text rows: they are dense and have no free candidate).
+ * margin[i] = distance of the deciding comparison from equality, relative to the total mass:
+ *             min(cum_k - target, target - cum_{k-1}) / total (+inf when tau >= 1 or no candidate).
+ * gap[i]    = as in oracle_select_mask: score of the last kept minus the best dropped candidate. */
+void oracle_select_mask_mass(const double *S, int nb, int n_text_blocks, double tau, double scale,
+                             uint8_t *mask /* [nb, nb] */, double *gap /* [nb] or NULL */,
+                             int32_t *k_out /* [nb] or NULL */, double *margin /* [nb] or NULL */) {
+    int *cand = (int *)malloc(sizeof(int) * (size_t)(nb > 0 ? nb : 1));
+    double *w = (double *)malloc(sizeof(double) * (size_t)(nb > 0 ? nb : 1));
+    for (int i = 0; i < nb; ++i) {
+        uint8_t *row = mask + (size_t)i * nb;
+        const double *Si = S + (size_t)i * nb;
+        memset(row, 0, (size_t)nb);
+        int nc = 0;
+        for (int j = 0; j < nb; ++j) {
+            int forced = (j < n_text_blocks) || (j == i) || (i < n_text_blocks);
+            if (forced) row[j] = 1; else cand[nc++] = j;
+        }
+        for (int a = 1; a < nc; ++a) {              /* order: score descending, index ascending */
+            int c = cand[a];
+            int b = a - 1;
+            while (b >= 0 && !(Si[cand[b]] > Si[c] || (Si[cand[b]] == Si[c] && cand[b] < c))) {
+                cand[b + 1] = cand[b];
+                --b;
+            }
+            cand[b + 1] = c;
+        }
+        int k = nc;
+        double mg = INFINITY;
+        if (nc > 0 && tau < 1.0) {
+            double total = 0.0;
+            for (int a = 0; a < nc; ++a) {
+                w[a] = exp(scale * (Si[cand[a]] - Si[cand[0]]));
+                total += w[a];
+            }
+            double target = tau * total, cum = 0.0;
+            k = nc;                                  /* rounding may leave the full sum a hair short of the target */
+            for (int a = 0; a < nc; ++a) {
+                double before = cum;
+                cum += w[a];
+                if (cum >= target) {
+                    double lo = target - before, hi = cum - target;
+                    k = a + 1;
+                    mg = (lo < hi ? lo : hi) / total;
+                    break;
+                }
+            }
+        }
+        for (int a = 0; a < k; ++a) row[cand[a]] = 1;
+        if (k_out) k_out[i] = k;
+        if (margin) margin[i] = mg;
+        if (gap) gap[i] = (k > 0 && k < nc) ? Si[cand[k - 1]] - Si[cand[k]] : INFINITY;
+    }
+    free(cand);
+    free(w);
+}
+
 /* Step 6: masked softmax attention of one (image, head) for query blocks [qb_lo, qb_hi).
  * For a query token n in block i, the keys are the valid tokens m of every block j with
  * mask[i, j] != 0;   z_m = scale * q_n . k_m;   p = softmax(z) over exactly those keys;
