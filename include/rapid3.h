@@ -108,6 +108,24 @@ int rapid3_select_mask(rapid3_ctx* ctx, const float* scores, const float* keep_r
                        uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, void* stream);
 
 /*
+ * Stage (a2), threshold variant (Sec. 3.2: the sparse candidates of the policy are thresholds of
+ * the sparse attention it drives, not counts; the rule itself is left to that method, so this is
+ * the plain cumulative-mass rule).  Forced blocks as in rapid3_select_mask.  For the free
+ * candidates c of a row, ordered by (score descending, index ascending), with weights
+ *     w_c = exp(mass_scale * (S[i][c] - max over the row's free candidates)),
+ * the row keeps the smallest number k >= 1 of leading candidates whose weights sum to at least
+ * mass_share_host[p] * (sum of all the row's weights); a share of exactly 1 keeps all of them.
+ * mass_share_host [n_img] (host) in (0, 1]; mass_scale >= 0, finite (e.g. the attention's softmax
+ * scale).  The weights and their sums are fp64 on the fp32 scores; scores must be finite.
+ * Outputs (device, caller-owned): row_keep [n_img, H, nb] int32 = k of every row (0 for text rows,
+ * which have no free candidate), and bitmask / kept_idx / kept_cnt as in rapid3_select_mask.
+ * Launches two kernels (the counts, then the selection at those counts).
+ */
+int rapid3_select_mask_mass(rapid3_ctx* ctx, const float* scores, const float* mass_share_host, float mass_scale,
+                            int n_img, int32_t* row_keep, uint64_t* bitmask, int32_t* kept_idx,
+                            int32_t* kept_cnt, void* stream);
+
+/*
  * Stage (b): masked flash-style attention over the kept tiles only.  For image p of the list
  * (batch index img_idx_host[p], or p when the list is NULL) the kept key blocks of query block
  * i are kept_idx[p][h][i][0 .. kept_cnt[p][h][i]).  kept_idx == NULL means every block is kept

@@ -22,7 +22,7 @@ EXPORTS = [
     "rapid3_create", "rapid3_destroy", "rapid3_strerror", "rapid3_num_blocks", "rapid3_mask_words",
     "rapid3_block_scores", "rapid3_select_mask", "rapid3_sparse_joint_attn", "rapid3_gated_step",
     "rapid3_gated_step_host", "rapid3_workspace", "rapid3_launch_count", "rapid3_last_status",
-    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device", "rapid3_gated_step_heads", "rapid3_equivalent_steps",
+    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device", "rapid3_gated_step_heads", "rapid3_equivalent_steps", "rapid3_select_mask_mass",
 ]
 
 
@@ -61,6 +61,7 @@ def load() -> ctypes.CDLL:
     lib.rapid3_mask_words.argtypes = [ctypes.POINTER(Shape)]
     lib.rapid3_block_scores.argtypes = [vp, vp, vp, i32p, ci, vp, vp]
     lib.rapid3_select_mask.argtypes = [vp, vp, f32p, ci, vp, vp, vp, vp]
+    lib.rapid3_select_mask_mass.argtypes = [vp, vp, f32p, cf, ci, vp, vp, vp, vp, vp]
     lib.rapid3_sparse_joint_attn.argtypes = [vp, vp, vp, vp, vp, i32p, ci, vp, vp, cf, vp]
     lib.rapid3_gated_step.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp]
     lib.rapid3_gated_step_heads.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp]
@@ -157,6 +158,20 @@ class Context:
         _check(self.lib.rapid3_select_mask(self.handle, _ptr(scores), _f32(keep_ratio), n, _ptr(bitmask),
                                            _ptr(kept_idx), _ptr(kept_cnt), _stream()), "rapid3_select_mask")
         return bitmask, kept_idx, kept_cnt
+
+    def rapid3_select_mask_mass(self, scores: torch.Tensor, mass_share: Sequence[float], mass_scale: float):
+        """Cumulative-mass selection: returns (row_keep, bitmask, kept_idx, kept_cnt)."""
+        n = scores.shape[0]
+        assert len(mass_share) == n and scores.dtype == torch.float32 and scores.is_contiguous()
+        dev = scores.device
+        row_keep = torch.empty((n, self.H, self.nb), dtype=torch.int32, device=dev)
+        bitmask = torch.empty((n, self.H, self.nb, self.words), dtype=torch.int64, device=dev)
+        kept_idx = torch.empty((n, self.H, self.nb, self.nb), dtype=torch.int32, device=dev)
+        kept_cnt = torch.empty((n, self.H, self.nb), dtype=torch.int32, device=dev)
+        _check(self.lib.rapid3_select_mask_mass(self.handle, _ptr(scores), _f32(mass_share), float(mass_scale), n,
+                                                _ptr(row_keep), _ptr(bitmask), _ptr(kept_idx), _ptr(kept_cnt),
+                                                _stream()), "rapid3_select_mask_mass")
+        return row_keep, bitmask, kept_idx, kept_cnt
 
     def rapid3_sparse_joint_attn(self, q, k, v, out, img_idx: Optional[Sequence[int]] = None,
                                  n_img: Optional[int] = None, kept_idx=None, kept_cnt=None,

@@ -298,6 +298,31 @@ int rapid3_select_mask(rapid3_ctx* c, const float* scores, const float* keep_rat
     return RAPID3_OK;
 }
 
+int rapid3_select_mask_mass(rapid3_ctx* c, const float* scores, const float* mass_share_host, float mass_scale,
+                            int n_img, int32_t* row_keep, uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt,
+                            void* stream) {
+    if (!c || !scores || !mass_share_host || !row_keep || !bitmask || !kept_idx || !kept_cnt) return RAPID3_ERR_INVALID_ARG;
+    if (!(mass_scale >= 0.f) || !isfinite(mass_scale)) return RAPID3_ERR_INVALID_ARG;
+    ImgList l;
+    int r = build_list(c, nullptr, n_img, &l);
+    if (r != RAPID3_OK) return r;
+    MassShare share;
+    for (int p = 0; p < n_img; ++p) {
+        const float tau = mass_share_host[p];
+        if (!(tau > 0.f) || !(tau <= 1.f)) return RAPID3_ERR_INVALID_ARG;
+        share.tau[p] = tau;
+        l.k_free[p] = 0;
+    }
+    {
+        ProfScope ps(c, PROF_SELECT, static_cast<cudaStream_t>(stream));
+        if (launch_select_mask_mass(scores, c->g, l, share, mass_scale, row_keep, bitmask, kept_idx, kept_cnt,
+                                    static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return RAPID3_ERR_CUDA;
+    }
+    c->launches += 2;
+    return RAPID3_OK;
+}
+
 int rapid3_sparse_joint_attn(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
                              const int32_t* img_idx_host, int n_img, const int32_t* kept_idx,
                              const int32_t* kept_cnt, float softmax_scale, void* stream) {

@@ -34,11 +34,21 @@ struct DevPlan {
 // sparsity head emits theta in R^{L x H}).  Travels as a kernel argument, so slots * H is bounded.
 #define RAPID3_MAX_HEAD_ROWS 2048
 struct HeadKeep {
-    static constexpr bool per_head = true;
+    static constexpr int mode = 1;
     int k[RAPID3_MAX_HEAD_ROWS];
 };
 struct NoHeadKeep {
-    static constexpr bool per_head = false;
+    static constexpr int mode = 0;
+};
+// Keep counts per row (image slot, head, query block) in device memory: the cumulative-mass rule
+// arrives at a different count in every row.
+struct RowKeep {
+    static constexpr int mode = 2;
+    const int32_t* k;
+};
+// Mass share tau per image of a launch (cumulative-mass selection).
+struct MassShare {
+    float tau[RAPID3_MAX_IMG];
 };
 
 struct TensorGeom {
@@ -61,6 +71,12 @@ cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const I
 cudaError_t launch_select_mask_heads(const float* scores, const TensorGeom& g, const ImgList& imgs,
                                      const HeadKeep& hk, uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt,
                                      cudaStream_t s);
+// K2, cumulative-mass variant: row_keep[row] = smallest count of best free candidates holding a share
+// tau of the row's softmax mass (weights exp(scale * (S - row max)), fp64), then the top-k selection
+// at that count.
+cudaError_t launch_select_mask_mass(const float* scores, const TensorGeom& g, const ImgList& imgs,
+                                    const MassShare& share, float scale, int32_t* row_keep, uint64_t* bitmask,
+                                    int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s);
 // Builds the plan from device-resident actions and keep ratios (one thread; B <= RAPID3_MAX_IMG).
 cudaError_t launch_plan(const int32_t* action_dev, const float* ratio_dev, int B, const TensorGeom& g,
                         DevPlan* plan, int* status, cudaStream_t s);

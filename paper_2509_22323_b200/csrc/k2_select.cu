@@ -13,7 +13,8 @@ namespace {
 
 constexpr int WARPS = 4;
 
-// HK = HeadKeep: one keep count per (image, head), passed by value.  HK = NoHeadKeep: per image.
+// HK = NoHeadKeep: one keep count per image.  HK = HeadKeep: one per (image, head), passed by value.
+// HK = RowKeep: one per row, read from device memory.
 template <typename HK>
 __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restrict__ scores, TensorGeom g,
                                                             ImgList imgs, uint32_t* __restrict__ bitmask32,
@@ -32,7 +33,8 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
     // free candidates kept in this row: one count per image, or per (image, head) when the policy
     // sets a ratio for every head
     int k;
-    if constexpr (HK::per_head) k = hk.k[p * g.H + (int)((row / nb) % g.H)];
+    if constexpr (HK::mode == 1) k = hk.k[p * g.H + (int)((row / nb) % g.H)];
+    else if constexpr (HK::mode == 2) k = hk.k[row];
     else k = plan ? plan->sparse.k_free[p] : imgs.k_free[p];
     uint32_t* s = reinterpret_cast<uint32_t*>(srow) + warp * nb_pad;
     const float* src = scores + row * nb;
@@ -104,7 +106,121 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
     if (lane == 0) kept_cnt[row] = total;
 }
 
+// Cumulative-mass rule: one warp per row finds the smallest count k of best free candidates (score
+// descending, index ascending) whose weights w = exp(scale * (S - row max)) sum to at least
+// tau * (sum of all free weights).  No sort: the boundary candidate is found by descending the
+// bits of the order-preserving keys, each round summing the weights of the candidates that match
+// the trial prefix (a weighted radix select); candidates equal to the boundary key are then added
+// one by one.  fp64 throughout, the precision in which the decision is defined.
+constexpr int MASS_WARPS = 2;
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__global__ void __launch_bounds__(MASS_WARPS * 32) mass_count_kernel(const float* __restrict__ scores, TensorGeom g,
+                                                                     int n_img, MassShare share, float scale,
+                                                                     int32_t* __restrict__ row_keep) {
+    extern __shared__ double mass_smem[];                  // [MASS_WARPS][nb_pad] weights, then the keys
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int nb = g.nb, ntb = g.n_text_blocks;
+    const int nb_pad = (nb + 31) & ~31;
+    const long long row = (long long)blockIdx.x * MASS_WARPS + warp;
+    if (row >= (long long)n_img * g.H * nb) return;
+    const int i = (int)(row % nb);
+    const int p = (int)(row / ((long long)nb * g.H));
+    const int n_free = (i < ntb) ? 0 : max(nb - ntb - 1, 0);
+    const float tau = share.tau[p];
+    if (n_free == 0 || tau >= 1.f) {                       // warp-uniform
+        if (lane == 0) row_keep[row] = n_free;
+        return;
+    }
+    double* w = mass_smem + warp * nb_pad;
+    uint32_t* key = reinterpret_cast<uint32_t*>(mass_smem + MASS_WARPS * nb_pad) + warp * nb_pad;
+    const float* src = scores + row * nb;
+    float mx = -INFINITY;
+    for (int j = lane; j < nb; j += 32)
+        if (j >= ntb && j != i) mx = fmaxf(mx, src[j]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    double part = 0.0;
+    for (int j = lane; j < nb_pad; j += 32) {
+        const bool is_free = j < nb && j >= ntb && j != i;
+        uint32_t u = 0u;
+        double wj = 0.0;
+        if (is_free) {
+            const float sj = src[j];
+            u = __float_as_uint(sj);
+            if (u == 0x80000000u) u = 0u;
+            u ^= (u >> 31) ? 0xffffffffu : 0x80000000u;
+            wj = exp((double)scale * ((double)sj - (double)mx));
+        }
+        key[j] = u;
+        w[j] = wj;                                         // forced and padding entries weigh nothing
+        part += wj;
+    }
+    __syncwarp();
+    const double total = warp_sum(part);
+    double want = (double)tau * total;                     // mass still to be covered inside the prefix group
+    uint32_t prefix = 0u, mask = 0u;
+    for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t trial = prefix | (1u << bit), m2 = mask | (1u << bit);
+        double m1 = 0.0;
+        for (int j = lane; j < nb_pad; j += 32) m1 += ((key[j] & m2) == trial) ? w[j] : 0.0;
+        m1 = warp_sum(m1);
+        if (m1 >= want) prefix = trial;
+        else want -= m1;
+        mask = m2;
+    }
+    // candidates above the boundary key are all kept; those equal to it one by one until the mass is reached
+    int n_gt = 0, n_eq = 0;
+    double w_eq = 0.0;
+    for (int j = lane; j < nb; j += 32) {
+        const bool is_free = j >= ntb && j != i;
+        n_gt += is_free && key[j] > prefix;
+        if (is_free && key[j] == prefix) {
+            ++n_eq;
+            w_eq = w[j];
+        }
+    }
+    n_gt = __reduce_add_sync(0xffffffffu, n_gt);
+    n_eq = __reduce_add_sync(0xffffffffu, n_eq);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) w_eq = fmax(w_eq, __shfl_xor_sync(0xffffffffu, w_eq, o));
+    int r = 0;
+    double acc = 0.0;
+    while (r < n_eq && (r == 0 || acc < want)) {
+        acc += w_eq;
+        ++r;
+    }
+    if (lane == 0) row_keep[row] = min(max(n_gt + r, 1), n_free);
+}
+
 }  // namespace
+
+cudaError_t launch_select_mask_mass(const float* scores, const TensorGeom& g, const ImgList& imgs,
+                                    const MassShare& share, float scale, int32_t* row_keep, uint64_t* bitmask,
+                                    int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s) {
+    const long long n_rows = (long long)imgs.n * g.H * g.nb;
+    const int nb_pad = (g.nb + 31) & ~31;
+    {
+        const unsigned grid = (unsigned)((n_rows + MASS_WARPS - 1) / MASS_WARPS);
+        const size_t smem = (size_t)MASS_WARPS * nb_pad * (sizeof(double) + sizeof(uint32_t));
+        mass_count_kernel<<<grid, MASS_WARPS * 32, smem, s>>>(scores, g, imgs.n, share, scale, row_keep);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    const int words32 = 2 * ((g.nb + 63) / 64);
+    const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
+    const size_t smem = (size_t)WARPS * nb_pad * sizeof(float);
+    RowKeep rk;
+    rk.k = row_keep;
+    select_kernel<RowKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
+                                                          kept_cnt, words32, nullptr, rk);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const ImgList& imgs, uint64_t* bitmask,
                                int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s, const DevPlan* plan, int n_cap) {
