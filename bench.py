@@ -386,6 +386,48 @@ def run_ours(args, wl):
             e["attention_speedup_vs_ratio_1"] = sweep[0]["attention_ms"] / e["attention_ms"]
             e["step_speedup_vs_ratio_1"] = sweep[0]["all_kernels_ms"] / e["all_kernels_ms"]
 
+    # the entry points beside the headline step, timed on the same inputs (device events, 20 calls each)
+    variants = None
+    if not args.no_sweep and wl.steps == 1:
+        variants = {}
+        (Q, K, V) = sets[0]
+        acts, ratios = plan[0][1], plan[0][2]
+
+        def timed(fn, n=20):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(n):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / n
+
+        # one keep ratio per (image, head): the image's ratio scaled by 0.5 / 1.0 / 1.5 in turn over the heads
+        head_ratios = [[min(1.0, r * (0.5 + 0.5 * (h % 3))) if r < 1.0 else 1.0 for h in range(wl.heads)] for r in ratios]
+        variants["gated_step_heads_ms"] = timed(lambda: ctx.rapid3_gated_step_heads(Q, K, V, out, acts, head_ratios,
+                                                                                  wl.softmax_scale))
+        variants["gated_step_ms"] = timed(lambda: ctx.rapid3_gated_step(Q, K, V, out, acts, ratios, wl.softmax_scale))
+        a_dev = torch.tensor(acts, dtype=torch.int32, device=dev)
+        r_dev = torch.tensor(ratios, dtype=torch.float32, device=dev)
+        variants["gated_step_device_ms"] = timed(lambda: ctx.rapid3_gated_step_device(Q, K, V, out, a_dev, r_dev,
+                                                                                    wl.softmax_scale))
+        n_sp = sum(1 for a, r in zip(acts, ratios) if a == binding.ACT_ATTEND and r < 1.0)
+        if n_sp:
+            sc = ctx.workspace(n_sp, device=dev)[0].clone()
+            variants["select_mask_mass_ms"] = timed(lambda: ctx.rapid3_select_mask_mass(sc, [0.5] * n_sp,
+                                                                                      4.0 * wl.softmax_scale))
+            variants["select_mask_ms"] = timed(lambda: ctx.rapid3_select_mask(sc, [0.5] * n_sp))
+            variants["select_images"] = n_sp
+        x = Q.reshape(wl.batch, -1)
+        o2, delta = torch.empty_like(x), torch.zeros_like(x)
+        cache_acts = [(binding.ACT_ATTEND, binding.ACT_REUSE)[b % 2] for b in range(wl.batch)]
+        ms = timed(lambda: binding.rapid3_cache_step(x, o2, delta, cache_acts))
+        variants["cache_step_ms"] = ms
+        variants["cache_step_gbs"] = 3 * x.numel() * 2 / (ms * 1e-3) / 1e9
+
     cpu = None
     if not args.no_cpu_baseline:
         v, secs, cores, desc = OracleSample(wl).run(args.cpu_budget)
@@ -401,7 +443,7 @@ def run_ours(args, wl):
                        "l2": f"inputs larger than L2 ({3 * sets[0][0].numel() * 2 / 1e6:.0f} MB per set), "
                              f"{nsets} input sets rotated"},
             "clocks": sampler.summary(w0, w1), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-            "cpu_baseline": cpu, "kernels": kernels, "keep_ratio_sweep": sweep}
+            "cpu_baseline": cpu, "kernels": kernels, "keep_ratio_sweep": sweep, "variants": variants}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
