@@ -60,6 +60,8 @@ def _load():
         lib.oracle_keep_count.restype = ci
         lib.oracle_select_mask.argtypes = [f64p, ci, ci, cd, u8p, f64p]
         lib.oracle_select_mask_mass.argtypes = [f64p, ci, ci, cd, cd, u8p, f64p, ctypes.POINTER(ctypes.c_int32), f64p]
+        lib.oracle_qk_prepare.argtypes = [u16p, ci, ci, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
+                                          cd, u16p]
         lib.oracle_masked_attention.argtypes = [u16p, u16p, u16p, ci, ci, u8p, cd, ci, ci, f64p]
         lib.oracle_attention_weights.argtypes = [u16p, u16p, ci, ci, u8p, cd, ci, f64p]
         lib.oracle_num_threads.restype = ci
@@ -279,3 +281,27 @@ def equivalent_steps(actions: Sequence[int], c_cache: Sequence[float], c_sparse:
         C_sparse = float(np.float32(cs)) if a == 2 else 0.0
         total += (1.0 - C_cache) * (1.0 - C_sparse)
     return total, int(np.floor(total + 0.5))
+
+
+# ----------------------------------------------------------------------------------------------
+# Q/K producer in front of the attention (RMS normalisation with a learned gain, then rotary
+# embedding, one rounding to bf16); see oracle_qk_prepare in the C file.
+
+def qk_prepare(x, gain: np.ndarray, rot: Optional[np.ndarray], eps: float) -> np.ndarray:
+    """x: [H, N, D] bf16 (or uint16 bits); gain: [D] fp32; rot: [N, D/2, 2] fp32 (cos, sin) or None.
+    Returns the bf16 bit patterns [H, N, D] (uint16)."""
+    xb = _bits(x)
+    H, N, D = xb.shape
+    gain = np.ascontiguousarray(gain, dtype=np.float32)
+    assert gain.shape == (D,)
+    rp = None
+    if rot is not None:
+        rot = np.ascontiguousarray(rot, dtype=np.float32)
+        assert rot.shape == (N, D // 2, 2)
+        rp = _p(rot, ctypes.c_float)
+    out = np.empty_like(xb)
+    lib = _load()
+    for h in range(H):
+        lib.oracle_qk_prepare(_p(xb[h], ctypes.c_uint16), N, D, _p(gain, ctypes.c_float), rp, float(eps),
+                              _p(out[h], ctypes.c_uint16))
+    return out

@@ -276,3 +276,46 @@ int oracle_num_threads(void) {
 #endif
     return n;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Q/K producer with the block pooling folded in (the step in front of the attention of an MMDiT
+ * block: per-head RMS normalisation of the projected queries / keys with a learned gain, then
+ * the rotary position embedding; the paper takes both from its base models and does not restate
+ * them).  For one [N, D] bf16 matrix (one image, one head), token n:
+ *     r      = 1 / sqrt(mean_d x[n, d]^2 + eps)
+ *     y[d]   = x[n, d] * r * gain[d]
+ *     z[2i]  = y[2i] cos(n, i) - y[2i+1] sin(n, i),   z[2i+1] = y[2i] sin(n, i) + y[2i+1] cos(n, i)
+ * with rot[n][i] = (cos, sin) given as fp32 numbers (NULL: no rotation); out = z rounded once
+ * to bf16, ties to even.  The block means the scoring pass needs are the means of the ROUNDED
+ * values, i.e. oracle_block_pool of `out`.  Arithmetic in fp64. */
+static uint16_t f64_to_bf16(double v) {
+    /* direct round-to-nearest-even of the 52-bit mantissa to 7 bits (no detour through fp32) */
+    uint64_t u;
+    memcpy(&u, &v, sizeof u);
+    uint16_t sign = (uint16_t)((u >> 63) << 15);
+    uint64_t mag = u & 0x7fffffffffffffffULL;
+    if (mag == 0) return sign;
+    mag += ((1ULL << 44) - 1) + ((mag >> 45) & 1);
+    int64_t e = (int64_t)(mag >> 52) - 1023 + 127;            /* exponent after a possible carry */
+    if (e <= 0) return sign;                                  /* below the bf16 normal range: zero */
+    if (e >= 255) return (uint16_t)(sign | 0x7f80);           /* infinity */
+    return (uint16_t)(sign | ((uint16_t)e << 7) | (uint16_t)((mag >> 45) & 0x7f));
+}
+
+void oracle_qk_prepare(const uint16_t *x, int N, int D, const float *gain /* [D] */,
+                       const float *rot /* [N, D/2, 2] or NULL */, double eps, uint16_t *out /* [N, D] */) {
+    double *y = (double *)malloc(sizeof(double) * (size_t)D);
+    for (int n = 0; n < N; ++n) {
+        double ss = 0.0;
+        for (int d = 0; d < D; ++d) { double v = bf16_to_f64(x[(size_t)n * D + d]); ss += v * v; }
+        double r = 1.0 / sqrt(ss / (double)D + eps);
+        for (int d = 0; d < D; ++d) y[d] = bf16_to_f64(x[(size_t)n * D + d]) * r * (double)gain[d];
+        for (int i = 0; i < D / 2; ++i) {
+            double c = 1.0, s = 0.0;
+            if (rot) { c = (double)rot[((size_t)n * (D / 2) + i) * 2]; s = (double)rot[((size_t)n * (D / 2) + i) * 2 + 1]; }
+            out[(size_t)n * D + 2 * i] = f64_to_bf16(y[2 * i] * c - y[2 * i + 1] * s);
+            out[(size_t)n * D + 2 * i + 1] = f64_to_bf16(y[2 * i] * s + y[2 * i + 1] * c);
+        }
+    }
+    free(y);
+}
