@@ -421,6 +421,30 @@ def run_ours(args, wl):
                                                                                       4.0 * wl.softmax_scale))
             variants["select_mask_ms"] = timed(lambda: ctx.rapid3_select_mask(sc, [0.5] * n_sp))
             variants["select_images"] = n_sp
+        # the gated step with the Q/K producer folded in (RMS norm, gain, rotary embedding, pooling): its
+        # first kernel replaces the pooling kernel; bytes = raw Q, K read + Q, K written for the attending images
+        gq = torch.ones(wl.head_dim, device=dev)
+        gk = torch.ones(wl.head_dim, device=dev)
+        # identity rotations (the inputs already carry their rotary embedding): the table is read like any
+        # other, and the block structure the masks depend on stays that of the workload
+        rot = torch.zeros((wl.n_tokens, wl.head_dim // 2, 2), device=dev)
+        rot[..., 0] = 1.0
+        q2, k2 = torch.empty_like(Q), torch.empty_like(K)
+        fused = lambda: ctx.rapid3_gated_step_fused(Q, K, V, gq, gk, rot, 1e-6, q2, k2, out, acts, ratios,
+                                                    wl.softmax_scale)
+        variants["gated_step_fused_ms"] = timed(fused)
+        ctx.profile(True)
+        ctx.profile_read()
+        for _ in range(20):
+            fused()
+        torch.cuda.synchronize()
+        pr = ctx.profile_read()
+        ctx.profile(False)
+        n_att = sum(1 for a in acts if a == binding.ACT_ATTEND)
+        prod_ms = pr["block_pool"][0] / pr["block_pool"][1]
+        variants["fused_step_kernels_ms"] = {kk: vv[0] / max(vv[1], 1) for kk, vv in pr.items()}
+        variants["producer_ms"] = prod_ms
+        variants["producer_gbs"] = n_att * 4 * wl.heads * wl.n_tokens * wl.head_dim * 2 / (prod_ms * 1e-3) / 1e9
         x = Q.reshape(wl.batch, -1)
         o2, delta = torch.empty_like(x), torch.zeros_like(x)
         cache_acts = [(binding.ACT_ATTEND, binding.ACT_REUSE)[b % 2] for b in range(wl.batch)]

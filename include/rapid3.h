@@ -165,6 +165,29 @@ int rapid3_gated_step_heads(rapid3_ctx* ctx, const void* q, const void* k, const
                             float softmax_scale, void* stream);
 
 /*
+ * The gated step with the producer of Q and K folded in (the paper takes the block in front of the
+ * attention from its base models: per-head RMS normalisation of the projected queries and keys
+ * with a learned gain, then the rotary position embedding).  One kernel reads q_raw / k_raw once,
+ * writes the finished bf16 q / k once and, for the images that will be scored, the block means of
+ * what it wrote: the separate pooling pass over Q and K of rapid3_gated_step (the only extra HBM
+ * pass the sparsity rule adds) is gone.  Per token row x[D] of an attending image:
+ *     r = 1 / sqrt(mean(x^2) + eps);   y[d] = x[d] * r * gain[d];
+ *     z[2i] = y[2i] cos - y[2i+1] sin,  z[2i+1] = y[2i] sin + y[2i+1] cos,  (cos, sin) = rot[n][i]
+ * rounded once to bf16 (fp32 arithmetic).  Then scoring, selection and attention run on q, k, v
+ * exactly as in rapid3_gated_step (4 launches with a sparse image, 2 without).
+ *   q_raw, k_raw, q, k : device, bf16, the context's [B, H, N, D] strides, 16-byte aligned;
+ *                        q may equal q_raw and k may equal k_raw (in place);
+ *   q_gain, k_gain     : device, fp32 [D], 16-byte aligned;
+ *   rot                : device, fp32 [N][D/2][2] = (cos, sin) per token and channel pair, 16-byte
+ *                        aligned, or NULL for no rotation;   eps >= 0.
+ * Rows of q, k and out that belong to gated images are not touched.
+ */
+int rapid3_gated_step_fused(rapid3_ctx* ctx, const void* q_raw, const void* k_raw, const void* v,
+                            const float* q_gain, const float* k_gain, const float* rot, float eps, void* q,
+                            void* k, void* out, const int32_t* action_host, const float* keep_ratio_host, int B,
+                            float softmax_scale, void* stream);
+
+/*
  * The same step with the policy's decisions left on the GPU (Sec. 3.3: the heads sample their
  * actions on the device; reading them back would cost a host synchronisation per step and layer):
  * action_dev [B] int32 and keep_ratio_dev [B] float are DEVICE arrays, read by the kernels when

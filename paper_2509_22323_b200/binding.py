@@ -22,7 +22,7 @@ EXPORTS = [
     "rapid3_create", "rapid3_destroy", "rapid3_strerror", "rapid3_num_blocks", "rapid3_mask_words",
     "rapid3_block_scores", "rapid3_select_mask", "rapid3_sparse_joint_attn", "rapid3_gated_step",
     "rapid3_gated_step_host", "rapid3_workspace", "rapid3_launch_count", "rapid3_last_status",
-    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device", "rapid3_gated_step_heads", "rapid3_equivalent_steps", "rapid3_select_mask_mass",
+    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device", "rapid3_gated_step_heads", "rapid3_equivalent_steps", "rapid3_select_mask_mass", "rapid3_gated_step_fused",
 ]
 
 
@@ -64,6 +64,7 @@ def load() -> ctypes.CDLL:
     lib.rapid3_select_mask_mass.argtypes = [vp, vp, f32p, cf, ci, vp, vp, vp, vp, vp]
     lib.rapid3_sparse_joint_attn.argtypes = [vp, vp, vp, vp, vp, i32p, ci, vp, vp, cf, vp]
     lib.rapid3_gated_step.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp]
+    lib.rapid3_gated_step_fused.argtypes = [vp, vp, vp, vp, vp, vp, vp, cf, vp, vp, vp, i32p, f32p, ci, cf, vp]
     lib.rapid3_gated_step_heads.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp]
     lib.rapid3_gated_step_device.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, cf, vp]
     lib.rapid3_gated_step_host.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp, i64p, i64p]
@@ -188,6 +189,19 @@ class Context:
         scale = softmax_scale if softmax_scale is not None else self.D ** -0.5
         _check(self.lib.rapid3_gated_step(self.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _i32(actions),
                                           _f32(keep_ratio), len(actions), scale, _stream()), "rapid3_gated_step")
+        return out
+
+    def rapid3_gated_step_fused(self, q_raw, k_raw, v, q_gain, k_gain, rot, eps: float, q, k, out,
+                                actions: Sequence[int], keep_ratio: Sequence[float],
+                                softmax_scale: Optional[float] = None):
+        """q_raw, k_raw -> (RMS norm, gain, rotary) -> q, k (may alias the raw tensors), then the gated step."""
+        scale = softmax_scale if softmax_scale is not None else self.D ** -0.5
+        assert q_gain.dtype == torch.float32 and k_gain.dtype == torch.float32
+        assert rot is None or (rot.dtype == torch.float32 and rot.is_contiguous())
+        _check(self.lib.rapid3_gated_step_fused(self.handle, _ptr(q_raw), _ptr(k_raw), _ptr(v), _ptr(q_gain),
+                                                _ptr(k_gain), _ptr(rot), float(eps), _ptr(q), _ptr(k), _ptr(out),
+                                                _i32(actions), _f32(keep_ratio), len(actions), scale, _stream()),
+               "rapid3_gated_step_fused")
         return out
 
     def rapid3_gated_step_heads(self, q, k, v, out, actions: Sequence[int], keep_ratio: Sequence[Sequence[float]],

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "librapid3.so")
-SOURCES = ["api.cu", "k1_scores.cu", "k2_select.cu", "k3_attn.cu", "k4_cache.cu"]
+SOURCES = ["api.cu", "k1_scores.cu", "k2_select.cu", "k3_attn.cu", "k4_cache.cu", "k5_prepare.cu"]
 HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "ptx.cuh"), os.path.join(ROOT, "include", "rapid3.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]

@@ -340,9 +340,11 @@ int rapid3_sparse_joint_attn(rapid3_ctx* c, const void* q, const void* k, const 
 
 // One gated step.  heads_per_ratio == 1: keep_ratio_host is [B].  heads_per_ratio == H: it is
 // [B][H], one ratio per (image, head); an image is dense only when all its heads keep everything.
+// With `prep` set, Q and K are first produced from prep->q_raw / k_raw into q / k by the fused
+// producer, which also writes the block means: the pooling kernel is then not launched.
 static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
                            const int32_t* action_host, const float* keep_ratio_host, int heads_per_ratio, int B,
-                           float softmax_scale, void* stream) {
+                           float softmax_scale, void* stream, const PrepArgs* prep = nullptr) {
     if (!c || !q || !k || !v || !out || !action_host || !keep_ratio_host) return RAPID3_ERR_INVALID_ARG;
     if (B < 1 || B > c->shape.B_max) return RAPID3_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return RAPID3_ERR_INVALID_ARG;
@@ -400,11 +402,17 @@ static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const vo
         ratio_of[pos] = ratio;
     }
     if (all.n == 0) return RAPID3_OK;                     // every image gated: nothing is launched
+    if (prep) {
+        ProfScope ps(c, PROF_POOL, st);
+        if (launch_prepare(*prep, c->g, all, sparse.n, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+        c->launches += 1;
+    }
     if (sparse.n > 0) {
         if ((reinterpret_cast<uintptr_t>(q) % 16) || (reinterpret_cast<uintptr_t>(k) % 16)) return RAPID3_ERR_INVALID_ARG;
-        {
+        if (!prep) {
             ProfScope ps(c, PROF_POOL, st);
             if (launch_block_pool(q, k, c->g, sparse, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+            c->launches += 1;
         }
         {
             ProfScope ps(c, PROF_SCORES, st);
@@ -417,7 +425,7 @@ static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const vo
                          : launch_select_mask(c->scores, c->g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st);
             if (e != cudaSuccess) return RAPID3_ERR_CUDA;
         }
-        c->launches += 3;
+        c->launches += 2;
     }
     return attn_launch(c, q, k, v, out, all, sparse.n ? c->kept_idx : nullptr, sparse.n ? c->kept_cnt : nullptr,
                        sparse.n ? c->bitmask : nullptr, softmax_scale, st);
@@ -427,6 +435,21 @@ int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v
                       const int32_t* action_host, const float* keep_ratio_host, int B, float softmax_scale,
                       void* stream) {
     return gated_step_impl(c, q, k, v, out, action_host, keep_ratio_host, 1, B, softmax_scale, stream);
+}
+
+int rapid3_gated_step_fused(rapid3_ctx* c, const void* q_raw, const void* k_raw, const void* v, const float* q_gain,
+                            const float* k_gain, const float* rot, float eps, void* q, void* k, void* out,
+                            const int32_t* action_host, const float* keep_ratio_host, int B, float softmax_scale,
+                            void* stream) {
+    if (!c || !q_raw || !k_raw || !q_gain || !k_gain || !q || !k) return RAPID3_ERR_INVALID_ARG;
+    if (!(eps >= 0.f) || !isfinite(eps)) return RAPID3_ERR_INVALID_ARG;
+    const uintptr_t al = reinterpret_cast<uintptr_t>(q_raw) | reinterpret_cast<uintptr_t>(k_raw) |
+                         reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k) |
+                         reinterpret_cast<uintptr_t>(q_gain) | reinterpret_cast<uintptr_t>(k_gain) |
+                         reinterpret_cast<uintptr_t>(rot);
+    if (al % 16) return RAPID3_ERR_INVALID_ARG;
+    PrepArgs prep{q_raw, k_raw, q, k, q_gain, k_gain, rot, eps};
+    return gated_step_impl(c, q, k, v, out, action_host, keep_ratio_host, 1, B, softmax_scale, stream, &prep);
 }
 
 int rapid3_gated_step_heads(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,

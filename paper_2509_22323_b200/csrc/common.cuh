@@ -77,6 +77,20 @@ cudaError_t launch_select_mask_heads(const float* scores, const TensorGeom& g, c
 cudaError_t launch_select_mask_mass(const float* scores, const TensorGeom& g, const ImgList& imgs,
                                     const MassShare& share, float scale, int32_t* row_keep, uint64_t* bitmask,
                                     int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s);
+// K5: Q/K producer (RMS norm + gain + rotary embedding -> bf16) that also writes the block means of
+// the images with a workspace slot.  pooled is [2][n_sparse][H][nb][D].
+struct PrepArgs {
+    const void* q_raw;
+    const void* k_raw;
+    void* q_out;
+    void* k_out;
+    const float* q_gain;
+    const float* k_gain;
+    const float* rot;     // [N][D/2][2] (cos, sin) or nullptr
+    float eps;
+};
+cudaError_t launch_prepare(const PrepArgs& a, const TensorGeom& g, const ImgList& imgs, int n_sparse, double* pooled,
+                           cudaStream_t s);
 // Builds the plan from device-resident actions and keep ratios (one thread; B <= RAPID3_MAX_IMG).
 cudaError_t launch_plan(const int32_t* action_dev, const float* ratio_dev, int B, const TensorGeom& g,
                         DevPlan* plan, int* status, cudaStream_t s);
