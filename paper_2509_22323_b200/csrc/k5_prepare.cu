@@ -106,10 +106,12 @@ __global__ void __launch_bounds__(128, PREP_MINB) prepare_kernel(const uint16_t*
             if (row < valid) {
                 *reinterpret_cast<uint4*>(dst + (long long)(n0 + row) * g.stride_n + c * 8) =
                     make_uint4(w[0], w[1], w[2], w[3]);
+                if (slot >= 0) {                              // only scored images need their block means
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    acc[2 * i] += (double)bf16_lo(w[i]);
-                    acc[2 * i + 1] += (double)bf16_hi(w[i]);
+                    for (int i = 0; i < 4; ++i) {
+                        acc[2 * i] += (double)bf16_lo(w[i]);
+                        acc[2 * i + 1] += (double)bf16_hi(w[i]);
+                    }
                 }
             }
         }
