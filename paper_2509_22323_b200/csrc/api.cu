@@ -196,7 +196,9 @@ int rapid3_create(rapid3_ctx** out, const rapid3_shape* shape) {
     g.nb = (g.N + 63) / 64;
     g.n_text_blocks = (shape->n_text + 63) / 64;
     // a 128 x 128 token grid after a block-aligned text prefix: one grid row = two blocks
-    g.pair_stride = (shape->n_image == 128 * 128 && shape->n_text % 64 == 0) ? 2 : 1;
+    // and when the text prefix is a whole number of quads, a quad is one column of four grid rows
+    g.pair_stride = 1;
+    if (shape->n_image == 128 * 128 && shape->n_text % 64 == 0) g.pair_stride = (g.n_text_blocks % 4 == 0) ? 3 : 2;
     g.stride_b = shape->stride_b;
     g.stride_h = shape->stride_h;
     g.stride_n = shape->stride_n;

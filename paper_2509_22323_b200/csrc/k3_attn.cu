@@ -136,8 +136,21 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     // Which two of the quad's four query blocks form a 128-row tile: neighbours (a, a + 1), or, when
     // a row of the image grid spans two blocks, vertical neighbours (a, a + 2), whose kept lists
     // overlap far more (measured on the 128 x 128 grid at keep ratio 0.25: 90 % against 63 % of
-    // the tile's MMA work lands on kept 64 x 64 sub-tiles)
+    // the tile's MMA work lands on kept 64 x 64 sub-tiles).
+    // pair_stride 3 goes further on that grid: the whole quad is one column of it -- members
+    // (b, b + 2, b + 4, b + 6), the left or the right halves of four consecutive grid rows -- so both
+    // tiles want nearly the same key blocks (union of the quad 98 instead of 134 blocks at keep ratio
+    // 0.25, both tiles busy on 68 % of them instead of 23 %).  qblk(a) is member a's query block.
     const bool ps2 = g.pair_stride == 2;
+    const bool vq = g.pair_stride == 3;
+    auto qblk = [&](int a) -> int {
+        int i = i0 + a;
+        if (vq && i >= g.n_text_blocks) {
+            const int r = i - g.n_text_blocks, w = r & 7;
+            i = g.n_text_blocks + (r & ~7) + ((w & 3) << 1) + (w >> 2);
+        }
+        return i;
+    };
 
     const uint32_t bQ = smem_u32(&ctl->q_full);
     const uint32_t bKF = smem_u32(&ctl->k_full[0]), bKE = smem_u32(&ctl->k_empty[0]);
@@ -188,7 +201,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             for (int dh = 0; dh < DH; ++dh)
                 tma_load_4d(sQ + (ps2 ? (a & 1) : (a >> 1)) * C::QTILE_BYTES + dh * QHALF_BYTES +
                                 (ps2 ? (a >> 1) : (a & 1)) * BLK_BYTES, &tmq, bQ,
-                            dh * 64, (i0 + a) * 64, h, b);
+                            dh * 64, qblk(a) * 64, h, b);
     }
 
     // ---------------------------------------------------------------- union of the four kept lists
@@ -198,12 +211,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     if (slot >= 0 && prm.bitmask32 != nullptr) {
         if (tid < 4 * nw) {
             const int a = tid / nw, w = tid - a * nw;
-            if (i0 + a < nb)
-                ctl->bm[a][w] = prm.bitmask32[(((long long)slot * g.H + h) * nb + i0 + a) * prm.words32 + w];
+            if (qblk(a) < nb)
+                ctl->bm[a][w] = prm.bitmask32[(((long long)slot * g.H + h) * nb + qblk(a)) * prm.words32 + w];
         }
     } else if (slot >= 0 && prm.kept_idx != nullptr) {
-        for (int a = 0; a < 4 && i0 + a < nb; ++a) {
-            const long long row = ((long long)slot * g.H + h) * nb + i0 + a;
+        for (int a = 0; a < 4 && qblk(a) < nb; ++a) {
+            const long long row = ((long long)slot * g.H + h) * nb + qblk(a);
             const int cnt = min(max(prm.kept_cnt[row], 0), nb);
             const int32_t* lst = prm.kept_idx + row * nb;
             for (int e = tid; e < cnt; e += NTHREADS) {
@@ -215,7 +228,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     } else if (tid < 32) {
         const int n = min(max(nb - tid * 32, 0), 32);
         const uint32_t val = n == 32 ? 0xffffffffu : ((1u << n) - 1u);
-        for (int a = 0; a < 4; ++a) ctl->bm[a][tid] = (i0 + a < nb) ? val : 0u;
+        for (int a = 0; a < 4; ++a) ctl->bm[a][tid] = (qblk(a) < nb) ? val : 0u;
     }
     __syncthreads();
     // one thread per key block: its position in the ascending union list is the number of union
@@ -522,11 +535,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         // the two warps of a query block meet, then one lane stores the block
         const int qb_id = a;
         named_barrier_sync(1 + qb_id, 64);
-        if (ok && (wl & 1) == 0 && lane == 0 && (i0 + qb_id) * 64 < N) {
+        if (ok && (wl & 1) == 0 && lane == 0 && qblk(qb_id) * 64 < N) {
 #pragma unroll
             for (int dh = 0; dh < DH; ++dh)
                 tma_store_4d(&tmo, sQ + t * C::QTILE_BYTES + dh * QHALF_BYTES + (wl >> 1) * BLK_BYTES, dh * 64,
-                             (i0 + qb_id) * 64, h, b);
+                             qblk(qb_id) * 64, h, b);
             bulk_commit_group();
             bulk_wait_read_all();
         }

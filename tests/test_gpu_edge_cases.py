@@ -96,3 +96,29 @@ def test_ratio_that_keeps_a_single_free_block():
     gpu_mask = binding.bitmask_to_dense(ctx.workspace(1)[1], wl.n_blocks).numpy()[0]
     parity.compare_masks(gpu_mask, ref["mask"], ref["gap"], "one_free")
     parity.compare_outputs(out[0], ref["out"], "one_free")
+
+
+@pytest.mark.parametrize("n_text,what", [(64, "vertical pairs inside consecutive quads (text prefix not a whole quad)"),
+                                         (256, "column quads (text prefix of one quad)")])
+def test_two_block_grid_rows_quad_layouts(n_text, what):
+    """A 128 x 128 token grid: one grid row spans two 64-token blocks and the kernel regroups the query
+    blocks of a CTA by grid column.  Both regroupings: masks of every row, attention on sampled query
+    blocks of both halves of a grid row, at the text boundary and at the end."""
+    wl = inputs.Workload("grid128", 1, 2, 64, n_text, 128, 8.0, (0.25,), rope=False, seed=49)
+    Q, K, V = inputs.make_qkv(wl, 0, device=DEV)
+    ctx = binding.Context(1, wl.heads, 64, n_text, wl.n_image)
+    out = poison(Q.shape)
+    ctx.rapid3_gated_step(Q, K, V, out, [2], [0.25], wl.softmax_scale)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    assert not (out.view(torch.int16) == np.int16(POISON)).any()
+    nb, ntb = wl.n_blocks, n_text // 64
+    ws = ctx.workspace(1)
+    dm = binding.bitmask_to_dense(ws[1], nb).numpy()
+    parity.check_lists(ws[2], ws[3], dm)
+    q, k, v = Q[0].cpu(), K[0].cpu(), V[0].cpu()
+    S32, mask, gap = oracle.image_mask(q, k, n_text, 0.25)
+    parity.compare_masks(dm[0], mask, gap, what)
+    qblocks = [0, ntb, ntb + 1, ntb + 2, ntb + 7, ntb + 8, ntb + 13, nb // 2, nb - 8, nb - 2, nb - 1]
+    ref = parity.oracle_out_samples(q, k, v, dm[0], wl.softmax_scale, [0, 1], qblocks)
+    parity.compare_outputs(out[0], ref, what)
