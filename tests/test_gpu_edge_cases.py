@@ -122,3 +122,61 @@ def test_two_block_grid_rows_quad_layouts(n_text, what):
     qblocks = [0, ntb, ntb + 1, ntb + 2, ntb + 7, ntb + 8, ntb + 13, nb // 2, nb - 8, nb - 2, nb - 1]
     ref = parity.oracle_out_samples(q, k, v, dm[0], wl.softmax_scale, [0, 1], qblocks)
     parity.compare_outputs(out[0], ref, what)
+
+
+def test_fused_producer_in_place_on_packed_projections():
+    """The fused step run in place on a packed [B, N, 3, H, D] projection buffer (the layout a fused QKV
+    projection writes): Q and K are normalised and rotated where they lie, V is read as it is."""
+    wl = inputs.Workload("packed_fused", 2, 3, 128, 77, 24, 2.0, (1.0, 0.4), rope=False, seed=42)
+    Q, K, V = inputs.make_qkv(wl, 0, device=DEV)
+    B, H, N, D = Q.shape
+    packed = torch.zeros((B, N, 3, H, D), dtype=torch.bfloat16, device=DEV)
+    for i, t in enumerate((Q * 3, K * 0.5, V)):
+        packed[:, :, i] = t.permute(0, 2, 1, 3)
+    q, k, v = (packed[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+    raw_q, raw_k = q.contiguous(), k.contiguous()
+    gen = torch.Generator(device="cpu").manual_seed(3)
+    gain = (0.5 + torch.rand(D, generator=gen)).to(DEV)
+    ang = torch.rand((N, D // 2), generator=gen, dtype=torch.float64) * 6.283185307179586
+    rot = torch.stack([torch.cos(ang), torch.sin(ang)], dim=-1).float().contiguous().to(DEV)
+    out = poison((B, H, N, D))
+    ctx = binding.Context(B, H, D, wl.n_text, wl.n_image, strides=q.stride()[:3])
+    ctx_out = binding.Context(B, H, D, wl.n_text, wl.n_image)             # contiguous twin for the comparison run
+    # the output has its own (contiguous) strides here, so it goes through a packed buffer as well
+    out_buf = poison((B, N, 3, H, D))
+    out_v = out_buf[:, :, 0].permute(0, 2, 1, 3)
+    ctx.rapid3_gated_step_fused(q, k, v, gain, gain, rot, 1e-6, q, k, out_v, [2, 2], list(wl.keep_ratios),
+                                wl.softmax_scale)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    for b in range(B):
+        for raw, got, name in ((raw_q, q, "Q"), (raw_k, k, "K")):
+            want = oracle.qk_prepare(raw[b].cpu(), gain.cpu().numpy(), rot.cpu().numpy(), 1e-6)
+            w = (want.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+            g = got[b].contiguous().to(torch.float64).cpu().numpy()
+            L = np.repeat(np.hypot(w[..., 0::2], w[..., 1::2]), 2, axis=-1)
+            assert (np.abs(g - w) <= np.abs(w) * 2.0 ** -7 + L * 2.0 ** -20).all(), f"{name} img {b}"
+            assert (g != w).mean() < 5e-3
+    assert torch.equal(packed[:, :, 2].permute(0, 2, 1, 3), V)              # V untouched
+    ctx_out.rapid3_gated_step(q.contiguous(), k.contiguous(), V, out, [2, 2], list(wl.keep_ratios), wl.softmax_scale)
+    torch.cuda.synchronize()
+    assert torch.equal(out_v.contiguous().view(torch.int16), out.view(torch.int16))
+
+
+def test_mass_selection_at_the_largest_sequence():
+    """1024 blocks: the weighted radix select of the cumulative-mass rule over 32 lane rounds per pass."""
+    wl = inputs.Workload("max_n_mass", 1, 1, 64, 0, 256, 8.0, (0.1,), rope=False, seed=44)
+    Q, K, V = inputs.make_qkv(wl, 0, device=DEV)
+    ctx = binding.Context(1, 1, 64, 0, wl.n_image)
+    scores = ctx.rapid3_block_scores(Q, K)
+    scale = 8.0 * wl.softmax_scale
+    row_keep, bitmask, kept_idx, kept_cnt = ctx.rapid3_select_mask_mass(scores, [0.3], scale)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    dm = binding.bitmask_to_dense(bitmask, 1024).numpy()
+    parity.check_lists(kept_idx, kept_cnt, dm)
+    S32, mask, gap, k, margin = oracle.image_mask_mass(Q[0].cpu(), K[0].cpu(), 0, 0.3, scale)
+    near = (margin <= 1e-9) | (gap <= parity.TIE_EPS)
+    assert not ((row_keep[0].cpu().numpy() != k) & ~near).any()
+    assert not ((dm[0] != mask).any(axis=-1) & ~near).any()
+    assert k.min() >= 1 and k.max() > k.min()
