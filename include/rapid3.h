@@ -239,9 +239,10 @@ int rapid3_workspace(rapid3_ctx* ctx, float** scores, uint64_t** bitmask, int32_
 int64_t rapid3_launch_count(rapid3_ctx* ctx);
 
 /*
- * Measurement aid (no counterpart in the paper): with profiling enabled every kernel launch of
- * this context is bracketed by a CUDA event pair on the caller's stream (at most 16384 pairs
- * between reads).  rapid3_profile_read waits for the recorded events, returns the summed device
+ * Measurement aid (no counterpart in the paper): with profiling enabled (enable = 1) every kernel
+ * launch of this context is bracketed by a CUDA event pair on the caller's stream (at most 16384
+ * pairs between reads); enable = 2 brackets the attention kernel only (an event pair costs a few
+ * microseconds of stream time, which matters beside the short scoring kernels); 0 switches it off.  rapid3_profile_read waits for the recorded events, returns the summed device
  * time in milliseconds and the launch count per kernel kind
  * (0 block pool, 1 block scores, 2 mask select, 3 attention) and clears the record.
  */

@@ -249,8 +249,9 @@ class Context:
     def launch_count(self) -> int:
         return int(self.lib.rapid3_launch_count(self.handle))
 
-    def profile(self, enable: bool):
-        _check(self.lib.rapid3_profile(self.handle, int(bool(enable))), "rapid3_profile")
+    def profile(self, enable):
+        """False / 0: off; True / 1: an event pair around every launch; 2: around the attention kernel only."""
+        _check(self.lib.rapid3_profile(self.handle, int(enable)), "rapid3_profile")
 
     def profile_read(self):
         """Summed device milliseconds and launch counts per kernel kind since the last read."""

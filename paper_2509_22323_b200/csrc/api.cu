@@ -49,7 +49,7 @@ struct rapid3_ctx {
     int map_rr = 0;
     int64_t launches = 0;
     // optional per-kernel timing (rapid3_profile): event pairs around each launch
-    bool prof_on = false;
+    int prof_mask = 0;            // bit k: launches of kernel kind k are bracketed by an event pair
     std::vector<ProfRec> prof;
     size_t prof_used = 0;
 };
@@ -64,7 +64,7 @@ struct ProfScope {
     cudaStream_t st;
     ProfRec* rec = nullptr;
     ProfScope(rapid3_ctx* ctx, int kind, cudaStream_t s) : c(ctx), st(s) {
-        if (!c->prof_on) return;
+        if (!((c->prof_mask >> kind) & 1)) return;
         if (c->prof_used == c->prof.size()) {
             if (c->prof.size() >= 16384) return;
             ProfRec r;
@@ -590,7 +590,8 @@ int64_t rapid3_launch_count(rapid3_ctx* c) { return c ? c->launches : -1; }
 
 int rapid3_profile(rapid3_ctx* c, int enable) {
     if (!c) return RAPID3_ERR_INVALID_ARG;
-    c->prof_on = enable != 0;
+    if (enable < 0 || enable > 2) return RAPID3_ERR_INVALID_ARG;
+    c->prof_mask = enable == 1 ? 0xF : (enable == 2 ? (1 << PROF_ATTN) : 0);
     return RAPID3_OK;
 }
 
