@@ -69,38 +69,69 @@ __global__ void __launch_bounds__(128) pool_kernel(const uint16_t* __restrict__ 
     }
 }
 
-// 32 x 32 tile of S per CTA, 16 x 16 threads, 2 x 2 outputs per thread, D in chunks of 32.
+// T x T tile of S per CTA (T = 32 or 64), 16 x 16 threads, (T/16) x (T/16) outputs per thread, D in
+// chunks of 32 staged in shared memory; the next chunk is fetched into registers while the current
+// one is multiplied.  Every output accumulates its D products in ascending channel order.
+template <int T>
 __global__ void __launch_bounds__(256) scores_kernel(const double* __restrict__ pooled, TensorGeom g, int n_img,
                                                      float* __restrict__ scores, const DevPlan* __restrict__ plan) {
-    __shared__ double sq[32][33];
-    __shared__ double sk[32][33];
+    constexpr int R = T / 16;            // outputs per thread and dimension
+    constexpr int LD = T * 32 / 256;     // values a thread stages per operand and chunk
+    __shared__ double sq[T][33];
+    __shared__ double sk[T][33];
     const int ph = blockIdx.z;                       // p * H + h
     if (plan && ph >= plan->sparse.n * g.H) return;
-    const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
+    const int i0 = blockIdx.y * T, j0 = blockIdx.x * T;
     const double* pq = pooled + (long long)ph * g.nb * g.D;
     const double* pk = pooled + ((long long)n_img * g.H + ph) * g.nb * g.D;
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
-    double a00 = 0, a01 = 0, a10 = 0, a11 = 0;
+    double acc[R][R];
+#pragma unroll
+    for (int a = 0; a < R; ++a)
+#pragma unroll
+        for (int b = 0; b < R; ++b) acc[a][b] = 0.0;
+    double rq[LD], rk[LD];
+    auto fetch = [&](int d0) {
+#pragma unroll
+        for (int u = 0; u < LD; ++u) {
+            const int e = threadIdx.x + u * 256, r = e / 32, c = e % 32;
+            rq[u] = (i0 + r < g.nb) ? pq[(long long)(i0 + r) * g.D + d0 + c] : 0.0;
+            rk[u] = (j0 + r < g.nb) ? pk[(long long)(j0 + r) * g.D + d0 + c] : 0.0;
+        }
+    };
+    fetch(0);
     for (int d0 = 0; d0 < g.D; d0 += 32) {
-        for (int e = threadIdx.x; e < 32 * 32; e += 256) {
-            int r = e / 32, c = e % 32;
-            sq[r][c] = (i0 + r < g.nb) ? pq[(long long)(i0 + r) * g.D + d0 + c] : 0.0;
-            sk[r][c] = (j0 + r < g.nb) ? pk[(long long)(j0 + r) * g.D + d0 + c] : 0.0;
+#pragma unroll
+        for (int u = 0; u < LD; ++u) {
+            const int e = threadIdx.x + u * 256, r = e / 32, c = e % 32;
+            sq[r][c] = rq[u];
+            sk[r][c] = rk[u];
         }
         __syncthreads();
+        if (d0 + 32 < g.D) fetch(d0 + 32);
 #pragma unroll 8
         for (int d = 0; d < 32; ++d) {
-            double q0 = sq[ty][d], q1 = sq[ty + 16][d], k0 = sk[tx][d], k1 = sk[tx + 16][d];
-            a00 += q0 * k0; a01 += q0 * k1; a10 += q1 * k0; a11 += q1 * k1;
+            double qv[R], kv[R];
+#pragma unroll
+            for (int a = 0; a < R; ++a) {
+                qv[a] = sq[ty + 16 * a][d];
+                kv[a] = sk[tx + 16 * a][d];
+            }
+#pragma unroll
+            for (int a = 0; a < R; ++a)
+#pragma unroll
+                for (int b = 0; b < R; ++b) acc[a][b] += qv[a] * kv[b];
         }
         __syncthreads();
     }
     float* so = scores + (long long)ph * g.nb * g.nb;
-    int i = i0 + ty, j = j0 + tx;
-    if (i < g.nb && j < g.nb) so[(long long)i * g.nb + j] = (float)a00;
-    if (i < g.nb && j + 16 < g.nb) so[(long long)i * g.nb + j + 16] = (float)a01;
-    if (i + 16 < g.nb && j < g.nb) so[(long long)(i + 16) * g.nb + j] = (float)a10;
-    if (i + 16 < g.nb && j + 16 < g.nb) so[(long long)(i + 16) * g.nb + j + 16] = (float)a11;
+#pragma unroll
+    for (int a = 0; a < R; ++a)
+#pragma unroll
+        for (int b = 0; b < R; ++b) {
+            const int i = i0 + ty + 16 * a, j = j0 + tx + 16 * b;
+            if (i < g.nb && j < g.nb) so[(long long)i * g.nb + j] = (float)acc[a][b];
+        }
 }
 
 }  // namespace
@@ -118,8 +149,15 @@ cudaError_t launch_block_pool(const void* q, const void* k, const TensorGeom& g,
 
 cudaError_t launch_block_scores(const double* pooled, const TensorGeom& g, int n_img, float* scores,
                                 cudaStream_t s, const DevPlan* plan) {
-    dim3 grid((g.nb + 31) / 32, (g.nb + 31) / 32, n_img * g.H);      // with a plan n_img is the capacity
-    scores_kernel<<<grid, 256, 0, s>>>(pooled, g, n_img, scores, plan);
+    // with a plan n_img is the capacity.  Long sequences take 64 x 64 tiles (half the shared-memory reads
+    // per product); short ones 32 x 32, which wastes less of the ragged edge and fills more SMs
+    if (g.nb >= 128) {
+        dim3 grid((g.nb + 63) / 64, (g.nb + 63) / 64, n_img * g.H);
+        scores_kernel<64><<<grid, 256, 0, s>>>(pooled, g, n_img, scores, plan);
+    } else {
+        dim3 grid((g.nb + 31) / 32, (g.nb + 31) / 32, n_img * g.H);
+        scores_kernel<32><<<grid, 256, 0, s>>>(pooled, g, n_img, scores, plan);
+    }
     return cudaGetLastError();
 }
 
