@@ -58,7 +58,7 @@ def test_small_configs_every_stage(name):
         # fp64 accumulation on both sides, one rounding to fp32: equal up to an occasional last-place flip
         np.testing.assert_allclose(scores[b].cpu().numpy(), S32, rtol=2e-7, atol=1e-9)
         flips = parity.compare_masks(gpu_mask[b], mask, gap, f"{name} img {b}")
-        # stage isolation: judge the attention against the oracle run with the GPU's own mask
+        # stage isolation: the attention is compared with the oracle run on the GPU's own mask
         ref = oracle.masked_attention(Qc[b], Kc[b], Vc[b], gpu_mask[b], wl.softmax_scale)
         parity.compare_outputs(out[b], ref, f"{name} img {b} ratio {ratio}")
         assert len(flips) == 0 or name != "tiny"
