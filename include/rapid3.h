@@ -165,6 +165,18 @@ int rapid3_gated_step_heads(rapid3_ctx* ctx, const void* q, const void* k, const
                             float softmax_scale, void* stream);
 
 /*
+ * The gated step with the cumulative-mass selection of rapid3_select_mask_mass in place of the
+ * top-k selection: mass_share_host[b] in (0, 1] is the share of attending image b (ignored for the
+ * others); a share of exactly 1 makes the image dense (no scoring); mass_scale as in
+ * rapid3_select_mask_mass.  Five launches with a sparse image (pool, scores, counts, selection,
+ * attention).  The per-row counts stay in the context's workspace.  Everything else as in
+ * rapid3_gated_step.
+ */
+int rapid3_gated_step_mass(rapid3_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                           const int32_t* action_host, const float* mass_share_host, float mass_scale, int B,
+                           float softmax_scale, void* stream);
+
+/*
  * The gated step with the producer of Q and K folded in (the paper takes the block in front of the
  * attention from its base models: per-head RMS normalisation of the projected queries and keys
  * with a learned gain, then the rotary position embedding).  One kernel reads q_raw / k_raw once,

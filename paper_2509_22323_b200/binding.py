@@ -22,7 +22,7 @@ EXPORTS = [
     "rapid3_create", "rapid3_destroy", "rapid3_strerror", "rapid3_num_blocks", "rapid3_mask_words",
     "rapid3_block_scores", "rapid3_select_mask", "rapid3_sparse_joint_attn", "rapid3_gated_step",
     "rapid3_gated_step_host", "rapid3_workspace", "rapid3_launch_count", "rapid3_last_status",
-    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device", "rapid3_gated_step_heads", "rapid3_equivalent_steps", "rapid3_select_mask_mass", "rapid3_gated_step_fused",
+    "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device", "rapid3_gated_step_heads", "rapid3_equivalent_steps", "rapid3_select_mask_mass", "rapid3_gated_step_fused", "rapid3_gated_step_mass",
 ]
 
 
@@ -65,6 +65,7 @@ def load() -> ctypes.CDLL:
     lib.rapid3_sparse_joint_attn.argtypes = [vp, vp, vp, vp, vp, i32p, ci, vp, vp, cf, vp]
     lib.rapid3_gated_step.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp]
     lib.rapid3_gated_step_fused.argtypes = [vp, vp, vp, vp, vp, vp, vp, cf, vp, vp, vp, i32p, f32p, ci, cf, vp]
+    lib.rapid3_gated_step_mass.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, cf, ci, cf, vp]
     lib.rapid3_gated_step_heads.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp]
     lib.rapid3_gated_step_device.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, cf, vp]
     lib.rapid3_gated_step_host.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp, i64p, i64p]
@@ -202,6 +203,15 @@ class Context:
                                                 _ptr(k_gain), _ptr(rot), float(eps), _ptr(q), _ptr(k), _ptr(out),
                                                 _i32(actions), _f32(keep_ratio), len(actions), scale, _stream()),
                "rapid3_gated_step_fused")
+        return out
+
+    def rapid3_gated_step_mass(self, q, k, v, out, actions: Sequence[int], mass_share: Sequence[float],
+                               mass_scale: float, softmax_scale: Optional[float] = None):
+        """The gated step with the cumulative-mass selection (share per image) instead of top-k."""
+        scale = softmax_scale if softmax_scale is not None else self.D ** -0.5
+        _check(self.lib.rapid3_gated_step_mass(self.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _i32(actions),
+                                               _f32(mass_share), float(mass_scale), len(actions), scale, _stream()),
+               "rapid3_gated_step_mass")
         return out
 
     def rapid3_gated_step_heads(self, q, k, v, out, actions: Sequence[int], keep_ratio: Sequence[Sequence[float]],

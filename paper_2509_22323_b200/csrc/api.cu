@@ -37,6 +37,7 @@ struct rapid3_ctx {
     uint64_t* bitmask = nullptr;  // [B_max][H][nb][words]
     int32_t* kept_idx = nullptr;  // [B_max][H][nb][nb]
     int32_t* kept_cnt = nullptr;  // [B_max][H][nb]
+    int32_t* row_keep = nullptr;  // [B_max][H][nb]: per-row counts of the cumulative-mass selection
     int* status = nullptr;
     DevPlan* plan = nullptr;      // device-resident plan of rapid3_gated_step_device
     // host-tensor staging of rapid3_gated_step_host (created on first use)
@@ -219,6 +220,7 @@ int rapid3_create(rapid3_ctx** out, const rapid3_shape* shape) {
               cudaMalloc(&c->bitmask, B * H * nb * c->words * sizeof(uint64_t)) == cudaSuccess &&
               cudaMalloc(&c->kept_idx, B * H * nb * nb * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&c->kept_cnt, B * H * nb * sizeof(int32_t)) == cudaSuccess &&
+              cudaMalloc(&c->row_keep, B * H * nb * sizeof(int32_t)) == cudaSuccess &&
               cudaMalloc(&c->status, sizeof(int)) == cudaSuccess &&
               cudaMemset(c->status, 0, sizeof(int)) == cudaSuccess &&
               cudaMalloc(&c->plan, sizeof(DevPlan)) == cudaSuccess &&
@@ -244,6 +246,7 @@ int rapid3_destroy(rapid3_ctx* c) {
     cudaFree(c->bitmask);
     cudaFree(c->kept_idx);
     cudaFree(c->kept_cnt);
+    cudaFree(c->row_keep);
     cudaFree(c->status);
     cudaFree(c->plan);
     for (void* s : c->stage) cudaFree(s);
@@ -346,7 +349,8 @@ int rapid3_sparse_joint_attn(rapid3_ctx* c, const void* q, const void* k, const 
 // producer, which also writes the block means: the pooling kernel is then not launched.
 static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
                            const int32_t* action_host, const float* keep_ratio_host, int heads_per_ratio, int B,
-                           float softmax_scale, void* stream, const PrepArgs* prep = nullptr) {
+                           float softmax_scale, void* stream, const PrepArgs* prep = nullptr,
+                           const float* mass_scale = nullptr) {
     if (!c || !q || !k || !v || !out || !action_host || !keep_ratio_host) return RAPID3_ERR_INVALID_ARG;
     if (B < 1 || B > c->shape.B_max) return RAPID3_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return RAPID3_ERR_INVALID_ARG;
@@ -358,9 +362,12 @@ static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const vo
     sparse.n = 0;
     all.n = 0;
     float ratio_of[RAPID3_MAX_IMG];
+    // with mass_scale set, keep_ratio_host holds mass shares and the selection is the cumulative-mass rule
     const bool per_head = heads_per_ratio > 1;
     const int H = c->g.H;
     HeadKeep hk;
+    MassShare share;
+    if (per_head) memset(&hk, 0, sizeof hk);
     for (int b = 0; b < B; ++b) {
         const int a = action_host[b];
         if (a != RAPID3_ACT_SKIP && a != RAPID3_ACT_REUSE && a != RAPID3_ACT_ATTEND) return RAPID3_ERR_INVALID_ARG;
@@ -384,6 +391,7 @@ static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const vo
             sparse.batch[slot] = b;
             sparse.slot[slot] = slot;
             sparse.k_free[slot] = keep_count((double)ratio, n_free_img > 0 ? n_free_img : 0);
+            share.tau[slot] = ratio;
             if (per_head) {
                 if ((slot + 1) * H > RAPID3_MAX_HEAD_ROWS) return RAPID3_ERR_UNSUPPORTED;
                 for (int h = 0; h < H; ++h)
@@ -423,11 +431,13 @@ static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const vo
         {
             ProfScope ps(c, PROF_SELECT, st);
             const cudaError_t e =
-                per_head ? launch_select_mask_heads(c->scores, c->g, sparse, hk, c->bitmask, c->kept_idx, c->kept_cnt, st)
-                         : launch_select_mask(c->scores, c->g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st);
+                mass_scale ? launch_select_mask_mass(c->scores, c->g, sparse, share, *mass_scale, c->row_keep, c->bitmask,
+                                                     c->kept_idx, c->kept_cnt, st)
+                : per_head ? launch_select_mask_heads(c->scores, c->g, sparse, hk, c->bitmask, c->kept_idx, c->kept_cnt, st)
+                           : launch_select_mask(c->scores, c->g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st);
             if (e != cudaSuccess) return RAPID3_ERR_CUDA;
         }
-        c->launches += 2;
+        c->launches += mass_scale ? 3 : 2;
     }
     return attn_launch(c, q, k, v, out, all, sparse.n ? c->kept_idx : nullptr, sparse.n ? c->kept_cnt : nullptr,
                        sparse.n ? c->bitmask : nullptr, softmax_scale, st);
@@ -437,6 +447,14 @@ int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v
                       const int32_t* action_host, const float* keep_ratio_host, int B, float softmax_scale,
                       void* stream) {
     return gated_step_impl(c, q, k, v, out, action_host, keep_ratio_host, 1, B, softmax_scale, stream);
+}
+
+int rapid3_gated_step_mass(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
+                           const int32_t* action_host, const float* mass_share_host, float mass_scale, int B,
+                           float softmax_scale, void* stream) {
+    if (!(mass_scale >= 0.f) || !isfinite(mass_scale)) return RAPID3_ERR_INVALID_ARG;
+    return gated_step_impl(c, q, k, v, out, action_host, mass_share_host, 1, B, softmax_scale, stream, nullptr,
+                           &mass_scale);
 }
 
 int rapid3_gated_step_fused(rapid3_ctx* c, const void* q_raw, const void* k_raw, const void* v, const float* q_gain,

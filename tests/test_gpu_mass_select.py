@@ -89,3 +89,33 @@ def test_mass_selection_full_size_masks(wl_name, shares):
         assert not ((row_keep[b] != k) & ~near).any()
         assert not ((gpu_mask[b] != mask).any(axis=-1) & ~near).any()
         print(f"{wl_name} img {b} share {tau}: counts {k[k > 0].min()}..{k.max()}, {int(near.sum())} near-tie rows")
+
+
+def test_gated_step_with_mass_selection():
+    """rapid3_gated_step_mass = gate + compaction + the staged mass path: same masks and outputs as the staged
+    calls on the attending images, gated images untouched, a share of 1 is dense."""
+    wl = inputs.Workload("mass_gate", 5, 2, 128, 64, 20, 2.0, (0.5,) * 5, rope=True, seed=73)
+    Q, K, V = inputs.make_qkv(wl, 0, device=DEV)
+    acts, shares = [2, 1, 2, 2, 0], [0.6, 0.5, 1.0, 0.2, 0.5]
+    scale = 4.0 * wl.softmax_scale
+    ctx = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
+    out = torch.full(Q.shape, 0x7FC1, dtype=torch.int16, device=DEV).view(torch.bfloat16)
+    n0 = ctx.launch_count()
+    ctx.rapid3_gated_step_mass(Q, K, V, out, acts, shares, scale, wl.softmax_scale)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0 and ctx.launch_count() - n0 == 5
+    raw = out.view(torch.int16)
+    assert (raw[1] == np.int16(0x7FC1)).all() and (raw[4] == np.int16(0x7FC1)).all()
+    ws = ctx.workspace(2)
+    gpu_mask = binding.bitmask_to_dense(ws[1], wl.n_blocks).numpy()
+    for slot, b in enumerate([0, 3]):
+        S32, mask, gap, k, margin = oracle.image_mask_mass(Q[b].cpu(), K[b].cpu(), wl.n_text, shares[b], scale)
+        near = (margin <= MARGIN_EPS) | (gap <= parity.TIE_EPS)
+        assert not ((gpu_mask[slot] != mask).any(axis=-1) & ~near).any()
+        ref = oracle.masked_attention(Q[b].cpu(), K[b].cpu(), V[b].cpu(), gpu_mask[slot], wl.softmax_scale)
+        parity.compare_outputs(out[b], ref, f"mass gate img {b}")
+    full = np.ones((wl.heads, wl.n_blocks, wl.n_blocks), np.uint8)
+    ref = oracle.masked_attention(Q[2].cpu(), K[2].cpu(), V[2].cpu(), full, wl.softmax_scale)
+    parity.compare_outputs(out[2], ref, "mass gate dense img 2")
+    with pytest.raises(binding.Rapid3Error):
+        ctx.rapid3_gated_step_mass(Q, K, V, out, acts, [0.6, 0.5, 1.0, 0.0, 0.5], scale)
