@@ -2,7 +2,8 @@
 // One warp per row.  The row of fp32 scores is staged in shared memory as order-preserving
 // 32-bit keys.  The k-th largest free candidate is found by a radix select over the key bits
 // (32 rounds of count-and-narrow, counts by lane-local sums and one warp reduction; rows with
-// fewer than ~100 candidates rank each candidate by counting instead); a free
+// fewer than ~100 candidates rank each candidate by counting the 64-bit (key, index) composites
+// that beat it instead); a free
 // candidate is kept when its key is above that threshold, or equal to it and among the first
 // (lowest block index) of the equal ones still needed -- the order "score descending, index
 // ascending".  The bitmask is assembled with warp ballots and the ascending kept list with ballot
@@ -21,7 +22,7 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
                                                             int32_t* __restrict__ kept_idx,
                                                             int32_t* __restrict__ kept_cnt, int words32,
                                                             const DevPlan* __restrict__ plan, const HK hk) {
-    extern __shared__ float srow[];                       // [WARPS][nb_pad]
+    extern __shared__ unsigned long long srow[];          // [WARPS][nb_pad] 64-bit slots
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int nb = g.nb, ntb = g.n_text_blocks;
     const int nb_pad = (nb + 31) & ~31;
@@ -36,31 +37,37 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
     if constexpr (HK::mode == 1) k = hk.k[p * g.H + (int)((row / nb) % g.H)];
     else if constexpr (HK::mode == 2) k = hk.k[row];
     else k = plan ? plan->sparse.k_free[p] : imgs.k_free[p];
-    uint32_t* s = reinterpret_cast<uint32_t*>(srow) + warp * nb_pad;
+    // long rows keep 32-bit keys in the slots' memory, short rows 64-bit (key, index) composites
+    unsigned long long* c64 = srow + warp * nb_pad;
+    uint32_t* s = reinterpret_cast<uint32_t*>(c64);
     const float* src = scores + row * nb;
     const bool text_row = i < ntb;
-    // key: unsigned integer with the same order as the float (-0 and +0 made equal)
+    const int n_free = max(nb - ntb - ((i >= ntb) ? 1 : 0), 0);
+    const bool select = !text_row && k > 0 && k < n_free;
+    const bool radix = n_free > 96;                     // short rows: ranking by counting is cheaper than 32 rounds
+    // key: unsigned integer with the same order as the float (-0 and +0 made equal), at least 2^23 for
+    // any finite score.  Forced blocks and padding get key 0: they match no radix prefix (every trial
+    // prefix has a bit set) and beat no candidate, so the loops below need no index tests.
     for (int j = lane; j < nb_pad; j += 32) {
         uint32_t u = 0u;
-        if (j < nb) {
+        if (j < nb && j >= ntb && j != i) {
             u = __float_as_uint(src[j]);
             if (u == 0x80000000u) u = 0u;
             u ^= (u >> 31) ? 0xffffffffu : 0x80000000u;
         }
-        s[j] = u;
+        // composite: equal scores rank by ascending block index, so no two candidates compare equal
+        if (radix) s[j] = u;
+        else c64[j] = u ? (((unsigned long long)u << 32) | (uint32_t)(0xffffffffu - (uint32_t)j)) : 0ull;
     }
     __syncwarp();
-    const int n_free = max(nb - ntb - ((i >= ntb) ? 1 : 0), 0);
     // radix select of the k-th largest key among the free candidates
     uint32_t prefix = 0u, mask = 0u;
     int want = k;                                       // rank still looked for inside the prefix group
-    const bool select = !text_row && k > 0 && k < n_free;
-    const bool radix = n_free > 96;                     // short rows: ranking by counting is cheaper than 32 rounds
     if (select && radix) {
         for (int bit = 31; bit >= 0; --bit) {
             const uint32_t trial = prefix | (1u << bit), m2 = mask | (1u << bit);
             int cnt = 0;
-            for (int j = lane; j < nb; j += 32) cnt += (j >= ntb) && (j != i) && ((s[j] & m2) == trial);
+            for (int j = lane; j < nb_pad; j += 32) cnt += ((s[j] & m2) == trial);
             cnt = __reduce_add_sync(0xffffffffu, cnt);
             if (cnt >= want) prefix = trial;
             else want -= cnt;
@@ -81,12 +88,10 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
                 eq = s[j] == prefix;
             } else if (select) {
                 // rank = number of free candidates that beat this one (key descending, index ascending)
-                const uint32_t sj = s[j];
+                const unsigned long long cj = c64[j];
                 int rank = 0;
-                for (int m = ntb; m < nb; ++m) {
-                    const uint32_t sm = s[m];
-                    rank += (m != i) && (sm > sj || (sm == sj && m < j));
-                }
+#pragma unroll 4
+                for (int m = ntb; m < nb; ++m) rank += c64[m] > cj;
                 keep = rank < k;
             } else {
                 keep = k >= n_free && k > 0;            // every free candidate, or none
@@ -214,7 +219,7 @@ cudaError_t launch_select_mask_mass(const float* scores, const TensorGeom& g, co
     }
     const int words32 = 2 * ((g.nb + 63) / 64);
     const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
-    const size_t smem = (size_t)WARPS * nb_pad * sizeof(float);
+    const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long);
     RowKeep rk;
     rk.k = row_keep;
     select_kernel<RowKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
@@ -228,7 +233,7 @@ cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const I
     const int nb_pad = (g.nb + 31) & ~31;
     const int words32 = 2 * ((g.nb + 63) / 64);
     const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
-    const size_t smem = (size_t)WARPS * nb_pad * sizeof(float);
+    const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long);
     select_kernel<NoHeadKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
                                                         kept_cnt, words32, plan, NoHeadKeep());
     return cudaGetLastError();
@@ -240,7 +245,7 @@ cudaError_t launch_select_mask_heads(const float* scores, const TensorGeom& g, c
     const int nb_pad = (g.nb + 31) & ~31;
     const int words32 = 2 * ((g.nb + 63) / 64);
     const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
-    const size_t smem = (size_t)WARPS * nb_pad * sizeof(float);
+    const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long);
     select_kernel<HeadKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
                                                        kept_cnt, words32, nullptr, hk);
     return cudaGetLastError();
