@@ -34,3 +34,27 @@ def test_strerror_and_shape_helpers_run_on_the_host():
     assert lib.rapid3_num_blocks(ctypes.byref(s2)) == 70
     bad = binding.Shape(1, 2, 96, 64, 256, 64, 1, 1, 96)
     assert lib.rapid3_num_blocks(ctypes.byref(bad)) == -2
+
+
+def test_null_context_is_refused_before_any_gpu_call():
+    """Every entry point that takes a context returns RAPID3_ERR_INVALID_ARG (-1) for a NULL one: host-side
+    argument checking runs before any CUDA call, so this holds without a GPU."""
+    import ctypes
+    lib = binding.load()
+    one_i = (ctypes.c_int32 * 1)(2)
+    one_f = (ctypes.c_float * 1)(0.5)
+    null = None
+    assert lib.rapid3_block_scores(null, null, null, null, 1, null, null) == -1
+    assert lib.rapid3_select_mask(null, null, one_f, 1, null, null, null, null) == -1
+    assert lib.rapid3_select_mask_mass(null, null, one_f, 1.0, 1, null, null, null, null, null) == -1
+    assert lib.rapid3_sparse_joint_attn(null, null, null, null, null, null, 1, null, null, 1.0, null) == -1
+    assert lib.rapid3_gated_step(null, null, null, null, null, one_i, one_f, 1, 1.0, null) == -1
+    assert lib.rapid3_gated_step_heads(null, null, null, null, null, one_i, one_f, 1, 1.0, null) == -1
+    assert lib.rapid3_gated_step_mass(null, null, null, null, null, one_i, one_f, 1.0, 1, 1.0, null) == -1
+    assert lib.rapid3_gated_step_device(null, null, null, null, null, null, null, 1, 1.0, null) == -1
+    assert lib.rapid3_gated_step_fused(null, null, null, null, null, null, null, 1e-6, null, null, null, one_i, one_f, 1,
+                                       1.0, null) == -1
+    assert lib.rapid3_gated_step_host(null, null, null, null, null, one_i, one_f, 1, 1.0, null, null, null) == -1
+    assert lib.rapid3_profile(null, 1) == -1
+    assert lib.rapid3_launch_count(null) == -1
+    assert lib.rapid3_destroy(null) in (0, -1)
