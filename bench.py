@@ -171,6 +171,32 @@ class OracleSample:
         return flops / secs / 1e12, secs, oracle.num_threads(), desc
 
 
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def oracle_tiny_single_thread():
+    """Seconds the oracle takes for the whole `tiny` workload on one thread (a child process, because the
+    OpenMP thread count is fixed when the oracle's library is loaded)."""
+    code = ("import time, oracle; from paper_2509_22323_b200 import inputs; wl = inputs.WORKLOADS['tiny'];"
+            "Q, K, V = inputs.make_qkv(wl, 0, device='cpu'); a, r = inputs.make_actions(wl, 0);"
+            "oracle.num_threads(); t = time.perf_counter();"
+            "oracle.gated_step(Q, K, V, a, r, wl.n_text, wl.softmax_scale); print(time.perf_counter() - t)")
+    try:
+        env = dict(os.environ, OMP_NUM_THREADS="1")
+        out = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=env, capture_output=True, text=True, timeout=300)
+        return float(out.stdout.strip().split()[-1])
+    except Exception:
+        return None
+
+
 def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -420,6 +446,13 @@ def run_ours(args, wl):
         variants["gated_step_heads_ms"] = timed(lambda: ctx.rapid3_gated_step_heads(Q, K, V, out, acts, head_ratios,
                                                                                   wl.softmax_scale))
         variants["gated_step_ms"] = timed(lambda: ctx.rapid3_gated_step(Q, K, V, out, acts, ratios, wl.softmax_scale))
+        # host time of one call through the Python binding (gate, compaction, four launches; nothing waits on the GPU)
+        torch.cuda.synchronize()
+        h0 = time.perf_counter()
+        for _ in range(100):
+            ctx.rapid3_gated_step(Q, K, V, out, acts, ratios, wl.softmax_scale)
+        variants["host_us_per_call"] = (time.perf_counter() - h0) / 100 * 1e6
+        torch.cuda.synchronize()
         a_dev = torch.tensor(acts, dtype=torch.int32, device=dev)
         r_dev = torch.tensor(ratios, dtype=torch.float32, device=dev)
         variants["gated_step_device_ms"] = timed(lambda: ctx.rapid3_gated_step_device(Q, K, V, out, a_dev, r_dev,
@@ -465,7 +498,8 @@ def run_ours(args, wl):
     cpu = None
     if not args.no_cpu_baseline:
         v, secs, cores, desc = OracleSample(wl).run(args.cpu_budget)
-        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "seconds": secs}
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "seconds": secs,
+               "cpu_model": cpu_model(), "tiny_1thread_seconds": oracle_tiny_single_thread()}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
