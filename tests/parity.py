@@ -43,8 +43,12 @@ def check_lists(kept_idx: torch.Tensor, kept_cnt: torch.Tensor, dense_mask: np.n
         assert (flat_i[r, flat_c[r]:] == -1).all()
 
 
-def compare_outputs(gpu_out: torch.Tensor, ora_out: np.ndarray, what: str = ""):
-    """gpu_out bf16 [..., N, D]; ora_out fp64 with NaN where the oracle was not evaluated."""
+def compare_outputs(gpu_out: torch.Tensor, ora_out: np.ndarray, what: str = "", scale_with_magnitude: bool = False):
+    """gpu_out bf16 [..., N, D]; ora_out fp64 with NaN where the oracle was not evaluated.
+    The two tolerances are absolute and presume outputs of a few units at most (the workloads' value
+    distribution).  With scale_with_magnitude they grow with the largest output: rounding the exact
+    result to bf16 alone costs up to 2^-8 of its magnitude (0.031 at |o| = 8), so for inputs that reach
+    |o| > 4 the bounds become 2^-7 max|o| and 2^-10 max|o|."""
     g = gpu_out.to(torch.float64).cpu().numpy()
     sel = ~np.isnan(ora_out)
     assert sel.any(), "nothing to compare"
@@ -52,8 +56,12 @@ def compare_outputs(gpu_out: torch.Tensor, ora_out: np.ndarray, what: str = ""):
     err = np.abs(g[sel] - ora_out[sel])
     mx, mean = float(err.max()), float(err.mean())
     print(f"{what}: max-abs {mx:.3e} mean-abs {mean:.3e} over {sel.sum()} values")
-    assert mx <= MAX_ABS_TOL, f"{what}: max-abs error {mx:.3e} > {MAX_ABS_TOL}"
-    assert mean <= MEAN_ABS_TOL, f"{what}: mean-abs error {mean:.3e} > {MEAN_ABS_TOL}"
+    max_tol, mean_tol = MAX_ABS_TOL, MEAN_ABS_TOL
+    if scale_with_magnitude:
+        big = float(np.abs(ora_out[sel]).max())
+        max_tol, mean_tol = max(max_tol, big * 2.0 ** -7), max(mean_tol, big * 2.0 ** -10)
+    assert mx <= max_tol, f"{what}: max-abs error {mx:.3e} > {max_tol}"
+    assert mean <= mean_tol, f"{what}: mean-abs error {mean:.3e} > {mean_tol}"
     return mx, mean
 
 
