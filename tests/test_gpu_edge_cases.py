@@ -180,3 +180,68 @@ def test_mass_selection_at_the_largest_sequence():
     assert not ((row_keep[0].cpu().numpy() != k) & ~near).any()
     assert not ((dm[0] != mask).any(axis=-1) & ~near).any()
     assert k.min() >= 1 and k.max() > k.min()
+
+
+def lists_from_mask(mask):
+    """[n, H, nb, nb] 0/1 -> (kept_idx int32 padded with -1, kept_cnt int32) in the library's layout."""
+    n, H, nb, _ = mask.shape
+    idx = np.full((n, H, nb, nb), -1, np.int32)
+    cnt = mask.sum(-1).astype(np.int32)
+    for p in range(n):
+        for h in range(H):
+            for i in range(nb):
+                js = np.nonzero(mask[p, h, i])[0]
+                idx[p, h, i, :len(js)] = js
+    return torch.from_numpy(idx).to(DEV), torch.from_numpy(cnt).to(DEV)
+
+
+@pytest.mark.parametrize("D,n_text,grid", [(128, 77, 20), (64, 0, 23)])
+def test_caller_supplied_lists_of_any_shape(D, n_text, grid):
+    """Kept lists the selection kernel would never write: rows that keep nothing (zero output), rows without
+    their diagonal or text blocks, single-block rows, whole quads that keep nothing, a full row."""
+    wl = inputs.Workload("anylist", 2, 2, D, n_text, grid, 2.0, (0.5, 0.5), seed=50)
+    Q, K, V = inputs.make_qkv(wl, 0, device=DEV)
+    nb = wl.n_blocks
+    rng = np.random.default_rng(12)
+    mask = (rng.random((2, 2, nb, nb)) < 0.3).astype(np.uint8)
+    mask[0, 0, 1] = 0                                    # a row that keeps nothing
+    mask[0, 1, 0:4] = 0                                  # a whole quad that keeps nothing
+    mask[1, 0, 2] = 0
+    mask[1, 0, 2, nb - 1] = 1                            # only the (ragged) last block
+    mask[1, 1, 3] = 1                                    # a full row
+    mask[1, 1, nb - 1] = 0
+    mask[1, 1, nb - 1, 0] = 1                            # the tail query block sees only block 0
+    kept_idx, kept_cnt = lists_from_mask(mask)
+    ctx = binding.Context(2, 2, D, n_text, wl.n_image)
+    out = poison(Q.shape)
+    ctx.rapid3_sparse_joint_attn(Q, K, V, out, kept_idx=kept_idx, kept_cnt=kept_cnt, softmax_scale=wl.softmax_scale)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    for b in range(2):
+        ref = oracle.masked_attention(Q[b].cpu(), K[b].cpu(), V[b].cpu(), mask[b], wl.softmax_scale)
+        parity.compare_outputs(out[b], ref, f"anylist img {b}")
+    o = out.float().cpu().numpy()
+    assert (o[0, 0, 64:128] == 0).all() and (o[0, 1, 0:256] == 0).all()          # nothing kept: exact zeros
+
+
+def test_malformed_list_sets_the_status_word_and_nothing_else():
+    wl = inputs.Workload("badlist", 1, 1, 64, 64, 12, 2.0, (0.5,), seed=51)
+    Q, K, V = inputs.make_qkv(wl, 0, device=DEV)
+    nb = wl.n_blocks
+    mask = np.ones((1, 1, nb, nb), np.uint8)
+    kept_idx, kept_cnt = lists_from_mask(mask)
+    kept_idx[0, 0, 1, 0] = nb + 5                        # out of range
+    kept_idx[0, 0, 2, 1] = -7                            # negative
+    kept_cnt[0, 0, 2] = nb + 100                         # count beyond the row (clamped)
+    ctx = binding.Context(1, 1, 64, 64, wl.n_image)
+    out = poison(Q.shape)
+    ctx.rapid3_sparse_joint_attn(Q, K, V, out, kept_idx=kept_idx, kept_cnt=kept_cnt, softmax_scale=wl.softmax_scale)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == -6                       # RAPID3_ERR_BAD_LIST, reported, no fault
+    assert ctx.last_status() == 0                        # reading clears it
+    assert torch.isfinite(out.float()).all()
+    # the rows with well-formed lists are what they should be
+    mask[0, 0, 1, 0] = 0
+    mask[0, 0, 2, 1] = 0
+    ref = oracle.masked_attention(Q[0].cpu(), K[0].cpu(), V[0].cpu(), mask[0], wl.softmax_scale, qb_lo=3, qb_hi=nb)
+    parity.compare_outputs(out[0], ref, "badlist rows 3..")
