@@ -245,3 +245,34 @@ def test_malformed_list_sets_the_status_word_and_nothing_else():
     mask[0, 0, 2, 1] = 0
     ref = oracle.masked_attention(Q[0].cpu(), K[0].cpu(), V[0].cpu(), mask[0], wl.softmax_scale, qb_lo=3, qb_hi=nb)
     parity.compare_outputs(out[0], ref, "badlist rows 3..")
+
+
+@pytest.mark.parametrize("D", [64, 128])
+def test_running_maximum_that_grows_with_every_key_block(D):
+    """Logits that climb from block to block by far more than the lazy-rescale threshold (and a very
+    sharp softmax): every block triggers the rescale of O and l.  Then the reverse order, where the
+    first block holds the maximum and everything after it underflows."""
+    wl = inputs.Workload("climb", 1, 2, D, 64, 16, 2.0, (1.0,), seed=52)
+    Q, K, V = inputs.make_qkv(wl, 0, device=DEV)
+    nb = wl.n_blocks
+    ramp = torch.arange(wl.n_tokens, device=DEV, dtype=torch.float32).div(64, rounding_mode="floor")
+    q0 = Q[0].float()
+    for direction in (1.0, -1.0):
+        # k_n = (3 * block(n) * direction) * unit vector along the mean query + small noise
+        u = q0.mean(dim=1, keepdim=True)
+        u = u / u.norm(dim=-1, keepdim=True)
+        Kc = (K[0].float() * 0.1 + direction * 3.0 * ramp[None, :, None] * u).to(torch.bfloat16)[None]
+        Qc = (q0 * 0.1 + 4.0 * u).to(torch.bfloat16)[None]
+        ctx = binding.Context(1, 2, D, 64, wl.n_image)
+        out = poison(Q.shape)
+        scale = 1.0                                             # logits step by about 12 per block: 2^17 in the exp2 domain
+        ctx.rapid3_sparse_joint_attn(Qc, Kc, V, out, softmax_scale=scale)
+        torch.cuda.synchronize()
+        assert ctx.last_status() == 0
+        full = np.ones((2, nb, nb), np.uint8)
+        ref = oracle.masked_attention(Qc[0].cpu(), Kc[0].cpu(), V[0].cpu(), full, scale)
+        parity.compare_outputs(out[0], ref, f"climb D={D} dir={direction}", scale_with_magnitude=True)
+        # the softmax really is that sharp: almost all the mass sits in one block
+        w = oracle.attention_weights(Qc[0].cpu(), Kc[0].cpu(), full, scale, 0, 100)
+        top = w.reshape(-1)[: (wl.n_tokens // 64) * 64].reshape(-1, 64).sum(-1).max()
+        assert top > 0.99
