@@ -276,3 +276,28 @@ def test_running_maximum_that_grows_with_every_key_block(D):
         w = oracle.attention_weights(Qc[0].cpu(), Kc[0].cpu(), full, scale, 0, 100)
         top = w.reshape(-1)[: (wl.n_tokens // 64) * 64].reshape(-1, 64).sum(-1).max()
         assert top > 0.99
+
+
+def test_two_contexts_on_two_streams():
+    """Two contexts driven from two streams at once (each owns its workspace and tensor maps): both give
+    what a single call gives."""
+    wl = inputs.Workload("streams", 3, 2, 128, 64, 24, 2.0, (1.0, 0.5, 0.25), rope=True, seed=53)
+    Q, K, V = inputs.make_qkv(wl, 0, device=DEV)
+    acts, ratios = [2, 2, 2], list(wl.keep_ratios)
+    ref_ctx = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
+    ref = poison(Q.shape)
+    ref_ctx.rapid3_gated_step(Q, K, V, ref, acts, ratios, wl.softmax_scale)
+    torch.cuda.synchronize()
+    ctxs = [binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image) for _ in range(2)]
+    outs = [poison(Q.shape) for _ in range(2)]
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    for rep in range(5):
+        for c, o, s in zip(ctxs, outs, streams):
+            with torch.cuda.stream(s):
+                c.rapid3_gated_step(Q, K, V, o, acts, ratios, wl.softmax_scale)
+    torch.cuda.synchronize()
+    for c, o in zip(ctxs, outs):
+        assert c.last_status() == 0
+        assert torch.equal(o.view(torch.int16), ref.view(torch.int16))
+        for a, b in zip(c.workspace(2), ref_ctx.workspace(2)):
+            assert torch.equal(a, b)
