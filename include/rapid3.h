@@ -144,6 +144,10 @@ int rapid3_sparse_joint_attn(rapid3_ctx* ctx, const void* q, const void* k, cons
  * passes.  Skipped and reusing images launch no work and their rows of `out` stay untouched.
  * Scores, masks and kept lists of the sparse images live in the context's workspace
  * (see rapid3_workspace), compacted in ascending batch order of the sparse images.
+ * The call only launches kernels (the tensor maps of a set of base pointers are encoded on the host at
+ * their first use and cached), so after one plain call with the same tensors it can be captured
+ * into a CUDA graph and replayed on buffers refilled in place; the actions and ratios are then
+ * those of the capture (rapid3_gated_step_device reads them on the GPU at every replay).
  */
 int rapid3_gated_step(rapid3_ctx* ctx, const void* q, const void* k, const void* v, void* out,
                       const int32_t* action_host, const float* keep_ratio_host, int B,

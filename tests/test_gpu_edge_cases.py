@@ -301,3 +301,30 @@ def test_two_contexts_on_two_streams():
         assert torch.equal(o.view(torch.int16), ref.view(torch.int16))
         for a, b in zip(c.workspace(2), ref_ctx.workspace(2)):
             assert torch.equal(a, b)
+
+
+def test_gated_step_inside_a_cuda_graph():
+    """The step makes no allocation, copy or synchronisation of its own, so it can be captured once and
+    replayed: the replays read the buffers' current contents (fresh Q, K, V written in place)."""
+    wl = inputs.Workload("graph", 3, 2, 128, 64, 20, 2.0, (1.0, 0.5, 0.25), rope=True, seed=54)
+    acts, ratios = [2, 2, 2], list(wl.keep_ratios)
+    ctx = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
+    Q, K, V = (t.clone() for t in inputs.make_qkv(wl, 0, device=DEV))
+    out = poison(Q.shape)
+    ctx.rapid3_gated_step(Q, K, V, out, acts, ratios, wl.softmax_scale)      # warm: tensor maps are encoded here
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ctx.rapid3_gated_step(Q, K, V, out, acts, ratios, wl.softmax_scale)
+    for step in (1, 2):
+        Qn, Kn, Vn = inputs.make_qkv(wl, step, device=DEV)
+        Q.copy_(Qn); K.copy_(Kn); V.copy_(Vn)
+        out.view(torch.int16).fill_(POISON)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ctx.last_status() == 0
+        want = poison(Q.shape)
+        ctx2 = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
+        ctx2.rapid3_gated_step(Qn, Kn, Vn, want, acts, ratios, wl.softmax_scale)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), want.view(torch.int16))
