@@ -57,3 +57,33 @@ def test_device_actions_flag_invalid_decisions():
     raw = out.view(torch.int16)
     assert not (raw[0] == np.int16(POISON)).any()                           # the valid image was processed
     assert (raw[1] == np.int16(POISON)).all() and (raw[2] == np.int16(POISON)).all()
+
+
+def test_device_actions_change_between_graph_replays():
+    """The point of device-resident decisions: one captured graph serves every step of a trajectory, the
+    policy writes new actions and ratios into the same device arrays between replays."""
+    wl = inputs.Workload("dev_graph", 4, 2, 128, 64, 20, 2.0, (0.5,) * 4, rope=True, seed=55)
+    Q, K, V = inputs.make_qkv(wl, 0, device=DEV)
+    ctx = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
+    a_dev = torch.tensor([2, 2, 2, 2], dtype=torch.int32, device=DEV)
+    r_dev = torch.tensor([0.5, 0.5, 0.5, 0.5], dtype=torch.float32, device=DEV)
+    out = poison_like(Q)
+    ctx.rapid3_gated_step_device(Q, K, V, out, a_dev, r_dev, wl.softmax_scale)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ctx.rapid3_gated_step_device(Q, K, V, out, a_dev, r_dev, wl.softmax_scale)
+    plans = [([2, 0, 2, 1], [1.0, 0.5, 0.25, 0.5]), ([0, 1, 0, 1], [0.5] * 4), ([2, 2, 2, 2], [0.1, 1.0, 1.0, 0.9]),
+             ([1, 2, 0, 0], [0.5, 0.3, 0.5, 0.5])]
+    for acts, ratios in plans:
+        a_dev.copy_(torch.tensor(acts, dtype=torch.int32))
+        r_dev.copy_(torch.tensor(ratios, dtype=torch.float32))
+        out.view(torch.int16).fill_(POISON)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ctx.last_status() == 0
+        want = poison_like(Q)
+        ctx_h = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
+        ctx_h.rapid3_gated_step(Q, K, V, want, acts, ratios, wl.softmax_scale)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), want.view(torch.int16)), (acts, ratios)
