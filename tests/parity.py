@@ -43,6 +43,19 @@ def check_lists(kept_idx: torch.Tensor, kept_cnt: torch.Tensor, dense_mask: np.n
         assert (flat_i[r, flat_c[r]:] == -1).all()
 
 
+def check_padding_bits(bitmask: torch.Tensor, nb: int):
+    """Bits at and beyond nb in the last word(s) of every bitmask row are zero."""
+    bm = bitmask.cpu().numpy().astype(np.uint64)
+    words = bm.shape[-1]
+    for w in range(words):
+        lo = 64 * w
+        if lo + 64 <= nb:
+            continue
+        valid = max(nb - lo, 0)
+        pad = np.uint64(0xFFFFFFFFFFFFFFFF) if valid == 0 else ~np.uint64((1 << valid) - 1)
+        assert not (bm[..., w] & pad).any(), f"bits >= {nb} set in word {w}"
+
+
 def compare_outputs(gpu_out: torch.Tensor, ora_out: np.ndarray, what: str = "", scale_with_magnitude: bool = False):
     """gpu_out bf16 [..., N, D]; ora_out fp64 with NaN where the oracle was not evaluated.
     The two tolerances are absolute and presume outputs of a few units at most (the workloads' value

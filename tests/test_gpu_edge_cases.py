@@ -59,6 +59,7 @@ def test_largest_sequence():
     ws = ctx.workspace(1)
     gpu_mask = binding.bitmask_to_dense(ws[1], 1024).numpy()[0]
     parity.check_lists(ws[2], ws[3], binding.bitmask_to_dense(ws[1], 1024).numpy())
+    parity.check_padding_bits(ws[1], 1024)
     q, k, v = Q[0].cpu(), K[0].cpu(), V[0].cpu()
     S32, mask, gap = oracle.image_mask(q, k, 0, 0.1)
     assert mask.sum(axis=-1).min() == 1 + 103          # diagonal + ceil(0.1 * 1023)

@@ -52,6 +52,7 @@ def test_small_configs_every_stage(name):
     assert ctx.nb == nb
     gpu_mask = binding.bitmask_to_dense(bitmask, nb).numpy()
     parity.check_lists(kept_idx, kept_cnt, gpu_mask)
+    parity.check_padding_bits(bitmask, nb)
     Qc, Kc, Vc = Q.cpu(), K.cpu(), V.cpu()
     for b, ratio in enumerate(wl.keep_ratios):
         S32, mask, gap = oracle.image_mask(Qc[b], Kc[b], wl.n_text, ratio)

@@ -40,6 +40,7 @@ def test_random_shape(seed):
         ws = ctx.workspace(len(sparse))
         dm = binding.bitmask_to_dense(ws[1], wl.n_blocks).numpy()
         parity.check_lists(ws[2], ws[3], dm)
+        parity.check_padding_bits(ws[1], wl.n_blocks)
         gpu_mask = {b: dm[s] for s, b in enumerate(sparse)}
     raw = out.view(torch.int16)
     for b in range(B):
