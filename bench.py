@@ -328,6 +328,7 @@ def run_ours(args, wl):
     torch.cuda.synchronize()
     prof_side = ctx.profile_read()
     ctx.profile(False)
+    assert ctx.last_status() == 0, "device status word is set after the timed region"
     for kind in ("block_pool", "block_scores", "select_mask"):
         prof[kind] = prof_side[kind]
     if rank == 0:
