@@ -222,9 +222,11 @@ int rapid3_gated_step_device(rapid3_ctx* ctx, const void* q, const void* k, cons
  * The same step with HOST tensors (pinned memory recommended): copies Q, K, V of the attending
  * images to device staging buffers, runs the step and copies their rows of `out` back; gated
  * images move no bytes.  The work is pipelined image by image over two copy streams owned by the
- * context (uploads of the next image, compute, downloads of the previous one overlap), forked
- * from and joined back into `stream`: seen from `stream` it is one ordered piece of work.  The
- * workspace afterwards describes the last sparse image processed only.  The staging buffers (4 tensors of
+ * context (uploads of the next image, compute, downloads of the previous one overlap; the last
+ * attending image goes in four groups of heads so that little is left to do after the last
+ * upload), forked from and joined back into `stream`: seen from `stream` it is one ordered piece
+ * of work.  The workspace afterwards describes the last piece processed only (the last head group
+ * of the last attending image, with that group's head count).  The staging buffers (4 tensors of
  * B_max*H*N*D bf16, contiguous [B, H, N, D]; the host tensors must be contiguous too) are
  * allocated on the first call of a context, so make that call outside any timed region.
  * bytes_h2d / bytes_d2h (may be NULL) receive the bytes moved.

@@ -58,6 +58,10 @@ struct rapid3_ctx {
 namespace {
 
 enum { PROF_POOL = 0, PROF_SCORES, PROF_SELECT, PROF_ATTN };
+#ifndef RAPID3_HOST_CHUNKS
+#define RAPID3_HOST_CHUNKS 4
+#endif
+constexpr int HOST_CHUNKS = RAPID3_HOST_CHUNKS;     // head groups per image in the host-tensor entry's pipeline
 
 // Records an event pair around one launch when profiling is on.
 struct ProfScope {
@@ -538,7 +542,7 @@ int rapid3_gated_step_host(rapid3_ctx* c, const void* q_host, const void* k_host
              cudaStreamCreateWithFlags(&c->down_s, cudaStreamNonBlocking) == cudaSuccess &&
              cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
              cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
-        for (int b = 0; b < s.B_max && ok; ++b) {
+        for (int b = 0; b < s.B_max * HOST_CHUNKS && ok; ++b) {
             cudaEvent_t e0 = nullptr, e1 = nullptr;
             ok = cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) == cudaSuccess &&
                  cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) == cudaSuccess;
@@ -554,39 +558,62 @@ int rapid3_gated_step_host(rapid3_ctx* c, const void* q_host, const void* k_host
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const void* src[3] = {q_host, k_host, v_host};
     int64_t up = 0, down = 0;
-    // Image by image: inputs go up on one copy stream, the step of that image runs on `stream` as soon
-    // as they have landed, its output goes down on a second copy stream -- so the uploads of the next
-    // images, the compute and the downloads overlap (the link is full duplex).  Everything is forked
-    // from and joined back into `stream`.
+    // Image by image: inputs go up on one copy stream, the step of that image runs on `stream` as soon as
+    // they have landed, its output goes down on a second copy stream -- so the uploads of the next images,
+    // the compute and the downloads overlap (the link is full duplex).  The last image goes in
+    // HOST_CHUNKS groups of heads (heads are independent), so that what is left after the last upload is
+    // one small group's compute and download.  Everything is forked from and joined back into `stream`.
     if (cudaEventRecord(c->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(c->up_s, c->ev_fork, 0) != cudaSuccess ||
         cudaStreamWaitEvent(c->down_s, c->ev_fork, 0) != cudaSuccess)
         return RAPID3_ERR_CUDA;
     int32_t one[RAPID3_MAX_IMG];
     for (int b = 0; b < B; ++b) one[b] = RAPID3_ACT_SKIP;
     bool any = false;
+    // only the last attending image is cut into head groups: every copy costs a few microseconds of
+    // engine turnaround, and it is the last image's compute and download that nothing overlaps
+    int last = -1;
+    for (int b = 0; b < B; ++b)
+        if (action_host[b] == RAPID3_ACT_ATTEND) last = b;
+    const int H_all = s.H;
+    const size_t head_bytes = (size_t)N * s.D * 2;
+    struct RestoreH {                                   // the kernels take the head count from the geometry
+        TensorGeom& g;
+        int H;
+        ~RestoreH() { g.H = H; }
+    } restore{c->g, H_all};
     for (int b = 0; b < B; ++b) {
         if (action_host[b] != RAPID3_ACT_ATTEND) continue;
         any = true;
-        for (int i = 0; i < 3; ++i) {
-            if (cudaMemcpyAsync((char*)c->stage[i] + b * img_bytes, (const char*)src[i] + b * img_bytes, img_bytes,
-                                cudaMemcpyHostToDevice, c->up_s) != cudaSuccess)
+        const int heads_per_chunk = (b == last) ? (H_all + HOST_CHUNKS - 1) / HOST_CHUNKS : H_all;
+        for (int h0 = 0, ch = 0; h0 < H_all; h0 += heads_per_chunk, ++ch) {
+            const int hn = (H_all - h0 < heads_per_chunk) ? H_all - h0 : heads_per_chunk;
+            const size_t off = b * img_bytes + h0 * head_bytes, bytes = hn * head_bytes;
+            cudaEvent_t e_up = c->ev_up[b * HOST_CHUNKS + ch], e_done = c->ev_done[b * HOST_CHUNKS + ch];
+            for (int i = 0; i < 3; ++i) {
+                if (cudaMemcpyAsync((char*)c->stage[i] + off, (const char*)src[i] + off, bytes, cudaMemcpyHostToDevice,
+                                    c->up_s) != cudaSuccess)
+                    return RAPID3_ERR_CUDA;
+                up += (int64_t)bytes;
+            }
+            if (cudaEventRecord(e_up, c->up_s) != cudaSuccess || cudaStreamWaitEvent(st, e_up, 0) != cudaSuccess)
                 return RAPID3_ERR_CUDA;
-            up += (int64_t)img_bytes;
+            // heads h0 .. h0 + hn of every tensor: the same strides from a base moved by h0 heads
+            one[b] = RAPID3_ACT_ATTEND;
+            c->g.H = hn;
+            const size_t hoff = h0 * head_bytes;
+            const int r = rapid3_gated_step(c, (char*)c->stage[0] + hoff, (char*)c->stage[1] + hoff,
+                                            (char*)c->stage[2] + hoff, (char*)c->stage[3] + hoff, one, keep_ratio_host, B,
+                                            softmax_scale, stream);
+            c->g.H = H_all;
+            one[b] = RAPID3_ACT_SKIP;
+            if (r != RAPID3_OK) return r;
+            if (cudaEventRecord(e_done, st) != cudaSuccess || cudaStreamWaitEvent(c->down_s, e_done, 0) != cudaSuccess)
+                return RAPID3_ERR_CUDA;
+            if (cudaMemcpyAsync((char*)out_host + off, (const char*)c->stage[3] + off, bytes, cudaMemcpyDeviceToHost,
+                                c->down_s) != cudaSuccess)
+                return RAPID3_ERR_CUDA;
+            down += (int64_t)bytes;
         }
-        if (cudaEventRecord(c->ev_up[b], c->up_s) != cudaSuccess || cudaStreamWaitEvent(st, c->ev_up[b], 0) != cudaSuccess)
-            return RAPID3_ERR_CUDA;
-        one[b] = RAPID3_ACT_ATTEND;
-        const int r = rapid3_gated_step(c, c->stage[0], c->stage[1], c->stage[2], c->stage[3], one, keep_ratio_host, B,
-                                        softmax_scale, stream);
-        one[b] = RAPID3_ACT_SKIP;
-        if (r != RAPID3_OK) return r;
-        if (cudaEventRecord(c->ev_done[b], st) != cudaSuccess ||
-            cudaStreamWaitEvent(c->down_s, c->ev_done[b], 0) != cudaSuccess)
-            return RAPID3_ERR_CUDA;
-        if (cudaMemcpyAsync((char*)out_host + b * img_bytes, (const char*)c->stage[3] + b * img_bytes, img_bytes,
-                            cudaMemcpyDeviceToHost, c->down_s) != cudaSuccess)
-            return RAPID3_ERR_CUDA;
-        down += (int64_t)img_bytes;
     }
     if (any && (cudaEventRecord(c->ev_join, c->down_s) != cudaSuccess || cudaStreamWaitEvent(st, c->ev_join, 0) != cudaSuccess))
         return RAPID3_ERR_CUDA;
