@@ -10,7 +10,8 @@
 //
 // Roles (352 threads):
 //   warp 8      producer: TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of Q once, then
-//               the gathered K and V blocks into two rings of shared-memory stages
+//               the gathered K and V blocks into two rings of shared-memory stages; K(g) and
+//               V(g - 1), which the MMA warps need together, complete one barrier
 //   warps 9,10  UMMA issue, one warp per tile (warp 9 also owns the TMEM allocation).  S of a
 //               tile is double buffered in TMEM (2 x 64 fp32 columns): S(n+1) = Q K^T is issued
 //               before O += P(n) V, so the tensor pipe works on the next scores while the
@@ -64,8 +65,8 @@ struct Cfg {
 
 struct __align__(16) Ctl {
     unsigned long long q_full;
-    unsigned long long k_full[MAX_STAGES], k_empty[MAX_STAGES];
-    unsigned long long v_full[MAX_STAGES], v_empty[MAX_STAGES];
+    unsigned long long k_full[MAX_STAGES], k_empty[MAX_STAGES];   // k_full[g % KS]: group g = K(g) and V(g - 1) have landed
+    unsigned long long v_empty[MAX_STAGES];
     unsigned long long s_full[2][2], p_full[2][2];
     unsigned long long pv_done[2], o_done[2], drain[2];
     uint32_t tmem_base;
@@ -154,7 +155,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
 
     const uint32_t bQ = smem_u32(&ctl->q_full);
     const uint32_t bKF = smem_u32(&ctl->k_full[0]), bKE = smem_u32(&ctl->k_empty[0]);
-    const uint32_t bVF = smem_u32(&ctl->v_full[0]), bVE = smem_u32(&ctl->v_empty[0]);
+    const uint32_t bVE = smem_u32(&ctl->v_empty[0]);
     const uint32_t bSF = smem_u32(&ctl->s_full[0][0]), bPF = smem_u32(&ctl->p_full[0][0]);   // [tile][buf]: + 16 t + 8 buf
     const uint32_t bPV = smem_u32(&ctl->pv_done[0]), bOD = smem_u32(&ctl->o_done[0]);        // [tile]: + 8 t
 
@@ -164,7 +165,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         for (int s = 0; s < MAX_STAGES; ++s) {
             mbar_init(bKF + 8 * s, 1);
             mbar_init(bKE + 8 * s, 2);      // both tiles pass a stage before it is refilled
-            mbar_init(bVF + 8 * s, 1);
             mbar_init(bVE + 8 * s, 2);
         }
         for (int s = 0; s < 4; ++s) {
@@ -276,42 +276,42 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
-            int k_issued = 0, v_issued = 0;
-            auto load_k = [&](int j) -> bool {
-                const int s = j % KS;
-                if (!wait(bKE + 8 * s, ((j / KS) & 1) ^ 1)) return false;
-                mbar_arrive_expect_tx(bKF + 8 * s, C::KV_BYTES);
-                const int blk = ctl->u_blk[j];
+            // Group g = K block g together with V block g - 1: the MMA warps need exactly that pair before they
+            // issue S(g) = Q K(g)^T and O += P(g-1) V(g-1), so the pair completes ONE barrier (g_full[g % KS]) and
+            // costs them one wait per key block instead of two.  Group 0 is K(0) alone, group n_u is V(n_u - 1)
+            // alone.  A group is armed once both ring stages it fills have been released.
+            int g_issued = 0;
+            auto load_group = [&](int gi) -> bool {
+                const int s = gi % KS;
+                const bool has_k = gi < n_u, has_v = gi > 0;
+                // the K stage's release also tells that both MMA warps are past their wait on this barrier's
+                // previous phase (group gi - KS), so it is awaited even when group n_u brings no K block
+                if (!wait(bKE + 8 * s, ((gi / KS) & 1) ^ 1)) return false;
+                const int jv = gi - 1, sv = has_v ? jv % VS : 0;
+                if (has_v && !wait(bVE + 8 * sv, ((jv / VS) & 1) ^ 1)) return false;
+                mbar_arrive_expect_tx(bKF + 8 * s, (has_k ? C::KV_BYTES : 0) + (has_v ? C::KV_BYTES : 0));
+                if (has_k) {
+                    const int blk = ctl->u_blk[gi];
 #pragma unroll
-                for (int dh = 0; dh < DH; ++dh)
-                    tma_load_4d(sK + s * C::KV_BYTES + dh * BLK_BYTES, &tmk, bKF + 8 * s, dh * 64, blk * 64, h, b);
-                k_issued = j + 1;
+                    for (int dh = 0; dh < DH; ++dh)
+                        tma_load_4d(sK + s * C::KV_BYTES + dh * BLK_BYTES, &tmk, bKF + 8 * s, dh * 64, blk * 64, h, b);
+                }
+                if (has_v) {
+                    const int blk = ctl->u_blk[jv];
+#pragma unroll
+                    for (int dh = 0; dh < DH; ++dh)
+                        tma_load_4d(sV + sv * C::KV_BYTES + dh * BLK_BYTES, &tmv, bKF + 8 * s, dh * 64, blk * 64, h, b);
+                }
+                g_issued = gi + 1;
                 return true;
             };
-            auto load_v = [&](int j) -> bool {
-                const int s = j % VS;
-                if (!wait(bVE + 8 * s, ((j / VS) & 1) ^ 1)) return false;
-                mbar_arrive_expect_tx(bVF + 8 * s, C::KV_BYTES);
-                const int blk = ctl->u_blk[j];
-#pragma unroll
-                for (int dh = 0; dh < DH; ++dh)
-                    tma_load_4d(sV + s * C::KV_BYTES + dh * BLK_BYTES, &tmv, bVF + 8 * s, dh * 64, blk * 64, h, b);
-                v_issued = j + 1;
-                return true;
-            };
-            // K runs one block ahead of V, the order in which the MMA warps consume them
-            bool ok = n_u > 0 ? load_k(0) : true;
-            for (int j = 0; ok && j < n_u; ++j) {
-                if (j + 1 < n_u && !(ok = load_k(j + 1))) break;
-                ok = load_v(j);
-            }
+            bool ok = true;
+            for (int gi = 0; ok && n_u > 0 && gi <= n_u; ++gi) ok = load_group(gi);
             if (ctl->abort_flag) {
                 // drain: do not leave the CTA while bulk copies may still land in its shared memory
                 mbar_wait(bQ, 0, 1u << 20);
-                for (int j = max(0, k_issued - KS); j < k_issued; ++j)
-                    mbar_wait(bKF + 8 * (j % KS), (j / KS) & 1, 1u << 20);
-                for (int j = max(0, v_issued - VS); j < v_issued; ++j)
-                    mbar_wait(bVF + 8 * (j % VS), (j / VS) & 1, 1u << 20);
+                for (int gi = max(0, g_issued - KS); gi < g_issued; ++gi)
+                    mbar_wait(bKF + 8 * (gi % KS), (gi / KS) & 1, 1u << 20);
             }
         }
         __syncwarp();
@@ -332,10 +332,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         constexpr uint32_t idesc_qk = idesc_bf16(128, 64, 0, 0);
         constexpr uint32_t idesc_pv = idesc_bf16(128, D, 0, 1);
         int n_qk = 0, n_pv = 0;                        // blocks of this tile issued so far
+        // waits for group gi (K(gi) and V(gi - 1), see the producer), then issues S = Q K(gi)^T
         auto k_step = [&](int j) -> bool {
             const int s = j % KS;
-            const bool use = ctl->u_flag[j] & tile_bits;
             if (!(wait_warp(bKF + 8 * s, (j / KS) & 1))) return false;
+            if (j >= n_u) return true;                 // the last group holds V(n_u - 1) only
+            const bool use = ctl->u_flag[j] & tile_bits;
             if (use) {
                 tc_fence_after();
                 const uint32_t tS = tbase + 64 * (n_qk & 1);
@@ -360,11 +362,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         for (int j = 0; ok && j < n_u; ++j) {
             // S(n+1) reuses the buffer of P(n-1); the MMAs of the issuing thread execute in issue
             // order, so it is written only after P(n-1) V has read it
-            if (j + 1 < n_u && !(ok = k_step(j + 1))) break;
+            if (!(ok = k_step(j + 1))) break;          // also brings V(j)
             const int s = j % VS;
             const bool use = ctl->u_flag[j] & tile_bits;
             if (use && !(ok = (wait_warp(bPFt + 8 * (n_pv & 1), (n_pv >> 1) & 1)))) break;
-            if (!(ok = (wait_warp(bVF + 8 * s, (j / VS) & 1)))) break;
             if (use) {
                 tc_fence_after();
                 const uint32_t tP = tbase + 64 * (n_pv & 1);
