@@ -35,6 +35,11 @@
  *     only the device can see (a bounded wait that ran out, a kept-list entry out of range)
  *     are recorded in a device status word, read with rapid3_last_status.
  *   - Non-finite inputs give undefined results.
+ *   - A context is used by one host thread at a time and its calls are ordered on the stream(s)
+ *     they are given: its workspace (block means, scores, masks, lists) is shared by all its
+ *     calls, so two calls of one context on different streams must be ordered by the caller.
+ *     Different contexts are independent (also on one device, on different streams) and a
+ *     context belongs to the device that was current when it was created.
  */
 #ifndef RAPID3_H_
 #define RAPID3_H_
