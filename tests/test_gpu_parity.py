@@ -167,3 +167,21 @@ def test_argument_errors_are_codes_not_faults():
         kw.update(bad)
         with pytest.raises(binding.Rapid3Error):
             binding.Context(**kw)
+
+
+def test_profile_modes_bracket_the_right_kernels():
+    wl = small_workload("prof", 2, 2, 64, 64, 12, 2.0, (0.5, 1.0))
+    Q, K, V = inputs.make_qkv(wl, 0, device=DEV)
+    ctx = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
+    out = poison_like(Q)
+    for mode, want in ((1, (3, 3, 3, 3)), (2, (0, 0, 0, 3)), (0, (0, 0, 0, 0))):
+        ctx.profile(mode)
+        ctx.profile_read()
+        for _ in range(3):
+            ctx.rapid3_gated_step(Q, K, V, out, [2, 2], [0.5, 1.0], wl.softmax_scale)
+        torch.cuda.synchronize()
+        pr = ctx.profile_read()
+        assert tuple(pr[k][1] for k in ("block_pool", "block_scores", "select_mask", "attention")) == want
+        assert all(pr[k][0] > 0 for k in pr if pr[k][1]) and all(pr[k][0] == 0 for k in pr if not pr[k][1])
+    with pytest.raises(binding.Rapid3Error):
+        ctx.profile(3)
