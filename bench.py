@@ -396,7 +396,7 @@ def run_ours(args, wl):
     # time of the same attention kernel at one keep ratio for the whole batch: ratio 1.0 is the dense
     # reference, the others show how the time follows the kept-tile fraction
     sweep = None
-    if not args.no_sweep and wl.steps == 1:
+    if not args.no_sweep and wl.steps == 1 and world == 1:
         sweep = []
         (Q, K, V) = sets[0]
         for r in (1.0, 0.5, 0.25):
@@ -425,7 +425,7 @@ def run_ours(args, wl):
 
     # the entry points beside the headline step, timed on the same inputs (device events, 20 calls each)
     variants = None
-    if not args.no_sweep and wl.steps == 1:
+    if not args.no_sweep and wl.steps == 1 and world == 1:
         variants = {}
         (Q, K, V) = sets[0]
         acts, ratios = plan[0][1], plan[0][2]
@@ -497,7 +497,7 @@ def run_ours(args, wl):
         variants["cache_step_gbs"] = 3 * x.numel() * 2 / (ms * 1e-3) / 1e9
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:          # the oracle is timed at N = 1 only
         v, secs, cores, desc = OracleSample(wl).run(args.cpu_budget)
         cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc, "seconds": secs,
                "cpu_model": cpu_model(), "tiny_1thread_seconds": oracle_tiny_single_thread()}
