@@ -34,7 +34,7 @@ METRIC = "block-sparse joint-attn ms/call & effective TFLOPS (kept tiles) vs bf1
 UNIT = "TFLOP/s (kept tiles)"
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu summary in
 # profiles/ (null until a capture of that workload exists)
-ATTN_DRAM_BYTES_PER_LAUNCH = {"flux_1024": 421726208, "flux_2048": 579465216, "sd3_1024": 93985536}
+ATTN_DRAM_BYTES_PER_LAUNCH = {"flux_1024": None, "flux_2048": None, "sd3_1024": None}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -123,7 +123,8 @@ class ClockSampler:
 # ----------------------------------------------------------------------------- CPU oracle legs
 class OracleSample:
     """The oracle (as it stands) on a bounded sample of the workload: mask selection of one sparse
-    image on all heads, plus attention on as many (head, query-block) units as fit the budget."""
+    image, then attention of WHOLE heads of that image (one oracle call per head over all its query
+    blocks, inputs converted to bit patterns once) until the time budget is used."""
 
     def __init__(self, wl, image=None):
         import oracle
@@ -133,41 +134,33 @@ class OracleSample:
             image = next((b for b, r in enumerate(wl.keep_ratios) if r < 1.0), 0)
         self.image = image
         self.ratio = wl.keep_ratios[image]
-        self.q, self.k, self.v = (inputs.make_tensor(wl, t, 0, image, "cpu") for t in range(3))
+        q, k, v = (inputs.make_tensor(wl, t, 0, image, "cpu") for t in range(3))
+        self.q, self.k, self.v = (np.ascontiguousarray(x.view(torch.int16).numpy().view(np.uint16)) for x in (q, k, v))
         nb = wl.n_blocks
         self.valid = np.full(nb, 64.0)
         self.valid[-1] = wl.n_tokens - 64 * (nb - 1)
-        # every (head, query-block) unit of the image in a fixed scattered order (stride coprime to
-        # the unit count), so that any prefix mixes text rows, image rows, the tail and all heads
-        n_units = wl.heads * nb
-        stride = next(s for s in range(max(2, int(0.618 * n_units)), 2 * n_units + 2) if np.gcd(s, n_units) == 1)
-        self.units = [divmod((u * stride) % n_units, nb) for u in range(n_units)]
 
     def run(self, budget_s, head=None):
-        """Returns (TFLOP/s on kept tiles, seconds, cores, description).  With `head` set, the
-        sample is that one head only (mask selection and attention units of that head)."""
+        """Returns (TFLOP/s on kept tiles, seconds, cores, description).  With `head` set the sample is
+        that one head; otherwise heads 0, 1, ... until `budget_s` seconds of attention have run."""
         wl, oracle = self.wl, self.oracle
         heads = list(range(wl.heads)) if head is None else [head]
-        q, k, v = (x[heads[0]:heads[-1] + 1] for x in (self.q, self.k, self.v))
-        t0 = time.perf_counter()
-        S32, mask, gap = oracle.image_mask(q, k, wl.n_text, self.ratio)
-        t_mask = time.perf_counter() - t0
-        flops, done, t_att = 0.0, 0, 0.0
-        for h, i in self.units:
-            if h not in heads:
-                continue
-            hl = h - heads[0]
-            t1 = time.perf_counter()
-            oracle.masked_attention(q, k, v, mask, wl.softmax_scale, qb_lo=i, qb_hi=i + 1, heads=[hl])
-            t_att += time.perf_counter() - t1
-            flops += 4.0 * wl.head_dim * self.valid[i] * float((mask[hl, i] * self.valid).sum())
+        flops, secs, done = 0.0, 0.0, 0
+        for h in heads:
+            q, k, v = self.q[h:h + 1], self.k[h:h + 1], self.v[h:h + 1]
+            t0 = time.perf_counter()
+            if self.ratio < 1.0:
+                _, mask, _ = oracle.image_mask(q, k, wl.n_text, self.ratio)
+            else:
+                mask = np.ones((1, wl.n_blocks, wl.n_blocks), np.uint8)
+            oracle.masked_attention(q, k, v, mask, wl.softmax_scale)
+            secs += time.perf_counter() - t0
+            flops += 4.0 * wl.head_dim * float((mask[0] * np.outer(self.valid, self.valid)).sum())
             done += 1
-            if t_att > budget_s:
+            if secs > budget_s:
                 break
-        # the mask pass covers every tile of the sampled heads; charge it in proportion to the sampled units
-        secs = t_att + t_mask * done / (len(heads) * wl.n_blocks)
-        desc = (f"{wl.name} image {self.image} (keep ratio {self.ratio}): mask selection on {len(heads)} head(s), "
-                f"attention on {done} sampled (head, query-block) units; mask time charged pro rata")
+        desc = (f"{wl.name} image {self.image} (keep ratio {self.ratio}): {done} whole head(s) of {wl.heads}, "
+                f"mask selection + attention over all {wl.n_blocks} query blocks of each")
         return flops / secs / 1e12, secs, oracle.num_threads(), desc
 
 
@@ -204,10 +197,9 @@ def run_reference(args, wl):
     sample = OracleSample(wl)
     vals, secs_all = [], []
     cores, desc = 0, ""
-    # every step is a bounded sample (one head, cycled); the whole run stays within ~2.5 minutes
-    budget = max(0.01, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
+    # every step is a bounded sample: one whole head (cycled) of one image
     for it in range(args.warmup + args.steps):
-        v, secs, cores, desc = sample.run(budget, head=it % wl.heads)
+        v, secs, cores, desc = sample.run(0.0, head=it % wl.heads)
         if it >= args.warmup:
             vals.append(v)
             secs_all.append(secs)
@@ -242,6 +234,212 @@ def aggregate(dist, device, ms_total: float, flops_total: float, launches: int):
 
 
 # ----------------------------------------------------------------------------- CUDA arm
+class Prepared:
+    """One workload ready to step: context, rotated input sets, per-step actions, and the kept-tile
+    flops of every step computed from the masks the library itself selected."""
+
+    def __init__(self, wl, rank, dev):
+        from paper_2509_22323_b200 import binding
+        self.binding, self.wl, self.dev = binding, wl, dev
+        self.ctx = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
+        nsets = 2
+        steps_of = list(range(nsets))
+        if wl.steps > 1:
+            steps_of = list(range(wl.steps))           # the gated trajectory: fresh Q/K/V per step
+            nsets = min(wl.steps, 4)
+        self.nsets = nsets
+        # inputs larger than L2 are rotated; small ones (the `tiny` workload) need an explicit flush
+        self.set_bytes = 3 * wl.batch * wl.heads * wl.n_tokens * wl.head_dim * 2
+        self.flush = torch.empty(192 << 20, dtype=torch.uint8, device=dev) if self.set_bytes * nsets < (160 << 20) else None
+        # each rank draws its own data (weak scaling): shift the step index by the rank
+        self.sets = [inputs.make_qkv(wl, rank_step(rank, st), device=dev) for st in range(nsets)]
+        self.out = torch.empty_like(self.sets[0][0])
+        self.plan = [(self.sets[i % nsets],) + tuple(inputs.make_actions(wl, steps_of[i % len(steps_of)]))
+                     for i in range(len(steps_of))]
+        self.flops_step, self.tiles_step = [], []
+        for i in range(len(self.plan)):
+            self.step(i)
+            torch.cuda.synchronize()
+            _, acts, ratios = self.plan[i]
+            sparse = [b for b, (a, r) in enumerate(zip(acts, ratios)) if a == binding.ACT_ATTEND and r < 1.0]
+            dense = [b for b, (a, r) in enumerate(zip(acts, ratios)) if a == binding.ACT_ATTEND and r >= 1.0]
+            masks = [(None, wl.heads)] * len(dense)
+            if sparse:
+                ws = self.ctx.workspace(len(sparse), device=dev)
+                dm = binding.bitmask_to_dense(ws[1], wl.n_blocks).numpy()
+                masks += [(dm[sl], wl.heads) for sl in range(len(sparse))]
+            f, t = kept_flops_from_masks(masks, wl.n_tokens, wl.head_dim)
+            self.flops_step.append(f)
+            self.tiles_step.append(t)
+        assert self.ctx.last_status() == 0, "device status word is set"
+
+    def step(self, i):
+        (Q, K, V), acts, ratios = self.plan[i % len(self.plan)]
+        if self.flush is not None:
+            self.flush.fill_(i & 0xFF)                 # evicts the small inputs from L2 between steps
+        self.ctx.rapid3_gated_step(Q, K, V, self.out, acts, ratios, self.wl.softmax_scale)
+
+    def flops(self, steps):
+        return sum(self.flops_step[i % len(self.plan)] for i in range(steps))
+
+    def l2_note(self):
+        if self.flush is not None:
+            return f"inputs smaller than L2: a {self.flush.numel() >> 20} MiB buffer is rewritten between steps"
+        return f"inputs larger than L2 ({self.set_bytes / 1e6:.0f} MB per set), {self.nsets} input sets rotated"
+
+
+def timed_region(pw, steps, warmup, dist=None):
+    """W warm-up steps, then K steps between one event pair (barrier + synchronize on both sides),
+    with an event pair around every attention launch inside.  Returns (ms_total, launches,
+    (attention ms, attention launches), wall-clock window)."""
+    ctx = pw.ctx
+    for i in range(warmup):
+        pw.step(i)
+    torch.cuda.synchronize()
+    ctx.profile(2)                     # an event pair around the attention kernel only: the roofline's duration
+    ctx.profile_read()
+    n0 = ctx.launch_count()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0 = time.time()
+    e0.record()
+    for i in range(steps):
+        pw.step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    w1 = time.time()
+    if dist is not None:
+        dist.barrier()
+    ms_total = e0.elapsed_time(e1)
+    launches = ctx.launch_count() - n0
+    attn = ctx.profile_read()["attention"]
+    ctx.profile(False)
+    return ms_total, launches, attn, (w0, w1)
+
+
+def per_step_times(pw, n):
+    """n further steps, each between its own event pair: median and minimum of the step time."""
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    torch.cuda.synchronize()
+    for i in range(n):
+        if pw.flush is not None:
+            pw.flush.fill_(i & 0xFF)
+        (Q, K, V), acts, ratios = pw.plan[i % len(pw.plan)]
+        evs[i].record()
+        pw.ctx.rapid3_gated_step(Q, K, V, pw.out, acts, ratios, pw.wl.softmax_scale)
+        evs[i + 1].record() if i == n - 1 else None
+    torch.cuda.synchronize()
+    # step i runs from its own record to the next step's record (the flush of a small workload sits before the record)
+    if pw.flush is None:
+        ts = [evs[i].elapsed_time(evs[i + 1]) for i in range(n)]
+    else:
+        ts = None
+    return ts
+
+
+def side_kernels(pw, n):
+    """Durations of all four kernels from a short pass with an event pair around every launch."""
+    pw.ctx.profile(1)
+    pw.ctx.profile_read()
+    for i in range(n):
+        pw.step(i)
+    torch.cuda.synchronize()
+    pr = pw.ctx.profile_read()
+    pw.ctx.profile(False)
+    return pr
+
+
+def attention_roofline(pw, steps, attn, ms_total, peaks, traffic):
+    attn_ms, attn_n = attn
+    attn_avg_ms = attn_ms / max(1, attn_n)
+    achieved = pw.flops(steps) / max(1, attn_n) / (attn_avg_ms * 1e-3) / 1e12 if attn_n else None
+    # a timed region under a second is a burst (clocks at their maximum, far below the power cap);
+    # a seconds-long one settles at the power cap, where the sustained GEMM figure is the fair peak
+    burst = ms_total < 1000.0
+    peak = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
+    which = "bf16_tflops" if burst else "bf16_tflops_sustained"
+    return {"bound": "tensor", "kernel": "attn_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+            "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+            "peak_source": f"{which} of {peaks['source']} (timed region {ms_total / 1e3:.3f} s: "
+                           f"{'burst' if burst else 'sustained'})",
+            "frac_of_burst_peak": (achieved / peaks["bf16_tflops"]) if achieved else None,
+            "frac_of_sustained_peak": (achieved / peaks["bf16_tflops_sustained"]) if achieved else None,
+            "frac_of_nominal_2250": (achieved / 2250.0) if achieved else None,
+            "avg_launch_ms": attn_avg_ms, "launches": attn_n}
+
+
+def keep_ratio_sweep(pw, n=20):
+    """The whole batch at one keep ratio: ratio 1.0 is the dense reference, the others show how the
+    time follows the kept-tile fraction."""
+    binding, wl, ctx = pw.binding, pw.wl, pw.ctx
+    (Q, K, V) = pw.sets[0]
+    sweep = []
+    for r in (1.0, 0.5, 0.25):
+        acts, ratios = [binding.ACT_ATTEND] * wl.batch, [r] * wl.batch
+        for _ in range(3):
+            ctx.rapid3_gated_step(Q, K, V, pw.out, acts, ratios, wl.softmax_scale)
+        torch.cuda.synchronize()
+        frac = 1.0
+        if r < 1.0:
+            frac = float(binding.bitmask_to_dense(ctx.workspace(wl.batch, device=pw.dev)[1], wl.n_blocks).numpy().mean())
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            ctx.rapid3_gated_step(Q, K, V, pw.out, acts, ratios, wl.softmax_scale)
+        b.record()
+        torch.cuda.synchronize()
+        step_ms = a.elapsed_time(b) / n
+        ctx.profile(True)
+        ctx.profile_read()
+        for _ in range(n):
+            ctx.rapid3_gated_step(Q, K, V, pw.out, acts, ratios, wl.softmax_scale)
+        torch.cuda.synchronize()
+        pr = ctx.profile_read()
+        ctx.profile(False)
+        sweep.append({"keep_ratio": r, "kept_tile_fraction": frac, "step_ms": step_ms,
+                      "attention_ms": pr["attention"][0] / pr["attention"][1],
+                      "kernels_ms_sum": sum(v[0] for v in pr.values()) / n})
+    for e in sweep:
+        e["attention_speedup_vs_ratio_1"] = sweep[0]["attention_ms"] / e["attention_ms"]
+        e["step_speedup_vs_ratio_1"] = sweep[0]["step_ms"] / e["step_ms"]
+        e["proportional_speedup"] = 1.0 / e["kept_tile_fraction"]
+    return sweep
+
+
+def workload_entry(name, peaks, steps=30, warmup=5):
+    """One line of the per-workload list: the same measurement as the headline, on another workload."""
+    wl = inputs.WORKLOADS[name]
+    dev = torch.device("cuda", torch.cuda.current_device())
+    pw = Prepared(wl, 0, dev)
+    if wl.steps > 1:
+        steps = 2 * wl.steps
+    ms_total, launches, attn, _ = timed_region(pw, steps, warmup)
+    roof = attention_roofline(pw, steps, attn, ms_total, peaks, None)
+    ts = per_step_times(pw, max(50, wl.steps * 2))
+    pr = side_kernels(pw, max(len(pw.plan), 20))
+    e = {"workload": name, "steps": steps, "ms_per_step": ms_total / steps,
+         "ms_per_step_median": statistics.median(ts) if ts else None, "ms_per_step_min": min(ts) if ts else None,
+         "attention_ms": roof["avg_launch_ms"], "value": pw.flops(steps) / (ms_total * 1e-3) / 1e12, "unit": UNIT,
+         "attention_tflops": roof["achieved"], "frac_of_burst_peak": roof["frac_of_burst_peak"],
+         "frac_of_nominal_2250": roof["frac_of_nominal_2250"], "gpu_launches": int(launches),
+         "kept_flops_per_step": pw.flops_step[0], "l2": pw.l2_note(),
+         "kernels_avg_ms": {k: (v[0] / v[1]) if v[1] else None for k, v in pr.items()}}
+    if wl.steps > 1:
+        per_traj = steps // wl.steps
+        e["ms_per_trajectory"] = ms_total / per_traj
+        e["launched_image_steps_per_trajectory"] = sum(
+            sum(1 for a in pw.plan[i][1] if a == pw.binding.ACT_ATTEND) for i in range(wl.steps))
+        e["kept_flops_per_trajectory"] = pw.flops(wl.steps)
+    elif name != "tiny":
+        e["keep_ratio_sweep"] = keep_ratio_sweep(pw)
+    assert pw.ctx.last_status() == 0, f"{name}: device status word is set"
+    del pw
+    torch.cuda.empty_cache()
+    return e
+
+
 def run_ours(args, wl):
     from paper_2509_22323_b200 import binding
 
@@ -258,84 +456,26 @@ def run_ours(args, wl):
         dist = dist_mod
         dist.init_process_group("nccl", device_id=dev)
 
-    ctx = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
-    nsets = 2
-    steps_of = list(range(nsets))
-    if wl.steps > 1:
-        steps_of = list(range(wl.steps))           # the gated trajectory: fresh Q/K/V per step
-        nsets = min(wl.steps, 4)
-    # each rank draws its own data (weak scaling): shift the step index by the rank
-    sets = [inputs.make_qkv(wl, rank_step(rank, s), device=dev) for s in range(nsets)]
-    out = torch.empty_like(sets[0][0])
-    plan = [(sets[i % nsets],) + tuple(inputs.make_actions(wl, steps_of[i % len(steps_of)])) for i in range(len(steps_of))]
-
-    def one_step(i):
-        (Q, K, V), acts, ratios = plan[i % len(plan)]
-        ctx.rapid3_gated_step(Q, K, V, out, acts, ratios, wl.softmax_scale)
-
-    # flops per step from the masks the library itself selected (marshalling for the report only)
-    flops_step, tiles_step, launches_img = [], [], []
-    for i in range(len(plan)):
-        one_step(i)
-        torch.cuda.synchronize()
-        (Q, K, V), acts, ratios = plan[i]
-        sparse = [b for b, (a, r) in enumerate(zip(acts, ratios)) if a == binding.ACT_ATTEND and r < 1.0]
-        dense = [b for b, (a, r) in enumerate(zip(acts, ratios)) if a == binding.ACT_ATTEND and r >= 1.0]
-        masks = [(None, wl.heads)] * len(dense)
-        if sparse:
-            ws = ctx.workspace(len(sparse), device=dev)
-            dm = binding.bitmask_to_dense(ws[1], wl.n_blocks).numpy()
-            masks += [(dm[s], wl.heads) for s in range(len(sparse))]
-        f, t = kept_flops_from_masks(masks, wl.n_tokens, wl.head_dim)
-        flops_step.append(f)
-        tiles_step.append(t)
-        launches_img.append(len(sparse) + len(dense))
-    assert ctx.last_status() == 0, "device status word is set"
-
-    for i in range(args.warmup):
-        one_step(i)
-    torch.cuda.synchronize()
+    pw = Prepared(wl, rank, dev)
+    ctx, sets, plan, out = pw.ctx, pw.sets, pw.plan, pw.out
+    flops_step, tiles_step = pw.flops_step, pw.tiles_step
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    ctx.profile(2)                     # an event pair around the attention kernel only: the roofline's duration
-    ctx.profile_read()
-    n0 = ctx.launch_count()
-    if dist is not None:
-        dist.barrier()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    w0 = time.time()
-    e0.record()
-    for i in range(args.steps):
-        one_step(i)
-    e1.record()
-    torch.cuda.synchronize()
-    w1 = time.time()
-    if dist is not None:
-        dist.barrier()
-    ms_total = e0.elapsed_time(e1)
-    launches = ctx.launch_count() - n0
-    prof = ctx.profile_read()
+    ms_total, launches, attn, (w0, w1) = timed_region(pw, args.steps, args.warmup, dist)
     # the other kernels' durations come from a short pass of their own (an event pair around every launch
     # costs a few microseconds of stream time each, which the timed region should not carry four times per step)
-    ctx.profile(1)
-    n_side = max(len(plan), min(args.steps, 50))
-    for i in range(n_side):
-        one_step(i)
-    torch.cuda.synchronize()
-    prof_side = ctx.profile_read()
-    ctx.profile(False)
+    prof = side_kernels(pw, max(len(plan), min(args.steps, 50)))
+    prof["attention"] = attn
+    step_ts = per_step_times(pw, max(50, 2 * len(plan)))
     assert ctx.last_status() == 0, "device status word is set after the timed region"
-    for kind in ("block_pool", "block_scores", "select_mask"):
-        prof[kind] = prof_side[kind]
     if rank == 0:
         time.sleep(0.2)
         sampler.stop()
-    flops_total = sum(flops_step[i % len(plan)] for i in range(args.steps))
-    ms_total, flops_total, launches = aggregate(dist, dev, ms_total, flops_total, launches)
+    rank_ms = ms_total
+    ms_total, flops_total, launches = aggregate(dist, dev, ms_total, pw.flops(args.steps), launches)
     value = flops_total / (ms_total * 1e-3) / 1e12
 
     # ---- end to end through the host-buffer entry point (rank-local, then max over ranks)
@@ -351,8 +491,10 @@ def run_ours(args, wl):
             dist.barrier()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a0.record()
+        h0 = time.perf_counter()
         for _ in range(n_e2e):
             up, down = ctx.rapid3_gated_step_host(hQ, hK, hV, hO, acts, ratios, wl.softmax_scale)
+        host_us = (time.perf_counter() - h0) / n_e2e * 1e6
         a1.record()
         torch.cuda.synchronize()
         ms_e2e = a0.elapsed_time(a1)
@@ -362,7 +504,7 @@ def run_ours(args, wl):
             ms_e2e = float(t.item())
         e2e = {"value": world * flops_step[0] * n_e2e / (ms_e2e * 1e-3) / 1e12, "unit": UNIT,
                "h2d_bytes_per_step": int(up), "d2h_bytes_per_step": int(down), "ms_per_step": ms_e2e / n_e2e,
-               "steps": n_e2e, "checksum": float(hO[0, 0, 0, :8].float().sum())}
+               "steps": n_e2e, "host_us_per_call": host_us, "checksum": float(hO[0, 0, 0, :8].float().sum())}
 
     if rank != 0:
         if dist is not None:
@@ -370,18 +512,7 @@ def run_ours(args, wl):
         return
 
     peaks = load_peaks()
-    attn_ms, attn_n = prof["attention"]
-    rank_flops = sum(flops_step[i % len(plan)] for i in range(args.steps))
-    attn_avg_ms = attn_ms / max(1, attn_n)
-    achieved = rank_flops / max(1, attn_n) / (attn_avg_ms * 1e-3) / 1e12 if attn_n else None
-    peak = peaks["bf16_tflops_sustained"]
-    traffic = ATTN_DRAM_BYTES_PER_LAUNCH.get(wl.name)
-    roofline = {"bound": "tensor", "kernel": "attn_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": (achieved / peak) if achieved else None, "traffic": traffic,
-                "peak_source": f"bf16_tflops_sustained of {peaks['source']}",
-                "frac_of_burst_peak": (achieved / peaks["bf16_tflops"]) if achieved else None,
-                "frac_of_nominal_2250": (achieved / 2250.0) if achieved else None,
-                "avg_launch_ms": attn_avg_ms, "launches": attn_n}
+    roofline = attention_roofline(pw, args.steps, attn, rank_ms, peaks, ATTN_DRAM_BYTES_PER_LAUNCH.get(wl.name))
     pool_ms, pool_n = prof["block_pool"]
     pool_bytes = None
     if pool_n:
@@ -393,35 +524,9 @@ def run_ours(args, wl):
         kernels["block_pool"]["achieved_gbs"] = pool_bytes / (pool_ms / pool_n * 1e-3) / 1e9
         kernels["block_pool"]["frac_of_hbm_peak"] = kernels["block_pool"]["achieved_gbs"] / peaks["hbm_gbs"]
 
-    # time of the same attention kernel at one keep ratio for the whole batch: ratio 1.0 is the dense
-    # reference, the others show how the time follows the kept-tile fraction
     sweep = None
     if not args.no_sweep and wl.steps == 1 and world == 1:
-        sweep = []
-        (Q, K, V) = sets[0]
-        for r in (1.0, 0.5, 0.25):
-            acts, ratios = [binding.ACT_ATTEND] * wl.batch, [r] * wl.batch
-            for _ in range(3):
-                ctx.rapid3_gated_step(Q, K, V, out, acts, ratios, wl.softmax_scale)
-            torch.cuda.synchronize()
-            if r < 1.0:
-                dm = binding.bitmask_to_dense(ctx.workspace(wl.batch, device=dev)[1], wl.n_blocks).numpy()
-                frac = float(dm.mean())
-            else:
-                frac = 1.0
-            ctx.profile(True)
-            ctx.profile_read()
-            for _ in range(20):
-                ctx.rapid3_gated_step(Q, K, V, out, acts, ratios, wl.softmax_scale)
-            torch.cuda.synchronize()
-            pr = ctx.profile_read()
-            ctx.profile(False)
-            step_ms = sum(v[0] for v in pr.values()) / 20.0
-            sweep.append({"keep_ratio": r, "kept_tile_fraction": frac, "attention_ms": pr["attention"][0] / pr["attention"][1],
-                          "all_kernels_ms": step_ms})
-        for e in sweep:
-            e["attention_speedup_vs_ratio_1"] = sweep[0]["attention_ms"] / e["attention_ms"]
-            e["step_speedup_vs_ratio_1"] = sweep[0]["all_kernels_ms"] / e["all_kernels_ms"]
+        sweep = keep_ratio_sweep(pw)
 
     # the entry points beside the headline step, timed on the same inputs (device events, 20 calls each)
     variants = None
@@ -495,6 +600,21 @@ def run_ours(args, wl):
         ms = timed(lambda: binding.rapid3_cache_step(x, o2, delta, cache_acts))
         variants["cache_step_ms"] = ms
         variants["cache_step_gbs"] = 3 * x.numel() * 2 / (ms * 1e-3) / 1e9
+        del q2, k2, o2, delta, rot
+
+    cfg_l2 = pw.l2_note()
+    del pw, ctx, sets, plan, out
+    torch.cuda.empty_cache()
+
+    # every workload of the configuration list on the same GPU in the same run (short regions: burst peak)
+    per_workload = None
+    if not args.no_per_workload and world == 1:
+        per_workload = []
+        for name in inputs.WORKLOADS:
+            try:
+                per_workload.append(workload_entry(name, peaks))
+            except Exception as exc:  # a failing side measurement must not lose the headline line
+                per_workload.append({"workload": name, "error": f"{type(exc).__name__}: {exc}"})
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:          # the oracle is timed at N = 1 only
@@ -503,19 +623,37 @@ def run_ours(args, wl):
                "cpu_model": cpu_model(), "tiny_1thread_seconds": oracle_tiny_single_thread()}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps,
+            "ms_per_step_median": statistics.median(step_ts) if step_ts else None,
+            "ms_per_step_min": min(step_ts) if step_ts else None,
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "batch": wl.batch, "heads": wl.heads, "head_dim": wl.head_dim,
                        "n_text": wl.n_text, "n_image": wl.n_image, "keep_ratios": list(wl.keep_ratios),
                        "trajectory_steps": wl.steps, "kept_tiles_per_step": tiles_step[0],
-                       "kept_flops_per_step": flops_step[0],
-                       "l2": f"inputs larger than L2 ({3 * sets[0][0].numel() * 2 / 1e6:.0f} MB per set), "
-                             f"{nsets} input sets rotated"},
+                       "kept_flops_per_step": flops_step[0], "l2": cfg_l2},
             "clocks": sampler.summary(w0, w1), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-            "cpu_baseline": cpu, "kernels": kernels, "keep_ratio_sweep": sweep, "variants": variants}
+            "cpu_baseline": cpu, "kernels": kernels, "keep_ratio_sweep": sweep, "variants": variants,
+            "per_workload": per_workload}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def spawn_ranks(args) -> int:
+    """`--gpus N` with N > 1 from a plain `python bench.py`: start N ranks of this script, one per GPU,
+    through torch.distributed.run on this node and pass their output through."""
+    import socket
+    n_dev = torch.cuda.device_count()
+    if n_dev < args.gpus:
+        sys.stderr.write(f"bench.py: --gpus {args.gpus} asked for, {n_dev} CUDA device(s) visible\n")
+        return 2
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -528,11 +666,17 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-per-workload", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     wl = inputs.WORKLOADS[args.workload]
+    world = int(os.environ.get("WORLD_SIZE", "0"))
+    if world == 0 and args.gpus > 1 and args.impl == "ours":
+        sys.exit(spawn_ranks(args))             # not under a launcher: start the N ranks here
+    if world > 0 and world != args.gpus:
+        sys.exit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world}")
     if args.impl == "reference":
         run_reference(args, wl)
     else:

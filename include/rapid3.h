@@ -54,7 +54,7 @@ typedef struct rapid3_ctx rapid3_ctx; /* opaque: workspace, tensor-map cache, st
 
 typedef struct rapid3_shape {
     int32_t B_max;    /* largest batch a call may pass (1..64)                        */
-    int32_t H;        /* heads                                                        */
+    int32_t H;        /* heads (B_max * H <= 65535, else RAPID3_ERR_UNSUPPORTED)      */
     int32_t D;        /* head dimension: 64 or 128                                    */
     int32_t n_text;   /* text tokens (>= 0), first in the joint sequence              */
     int32_t n_image;  /* image tokens (>= 0), after the text tokens; N = n_text+n_image, 1..65536 */
@@ -317,6 +317,21 @@ int rapid3_equivalent_steps(const int32_t* action_host, const float* c_cache_hos
 /* Copies the device status word to *device_status (RAPID3_OK or a negative code) and clears it.
  * Synchronises the device; call it after the stream has been synchronised. */
 int rapid3_last_status(rapid3_ctx* ctx, int* device_status);
+
+/*
+ * Test aid for the failure path (no counterpart in the paper; not part of the hot path).
+ * Launches a separately compiled failure-injection build of the attention kernel as a dense
+ * attention over image 0 of q, k, v: its producer stops issuing copies before group `stop_group`
+ * (group g = key block g together with value block g - 1; 0 <= stop_group <= nb), and every
+ * barrier wait in it gives up after 4096 polls instead of 2^22.  The waits of the other roles
+ * therefore run out: each thread block records RAPID3_ERR_TIMEOUT in the status word, waits
+ * (bounded) for its copies in flight, lets its tensor-core work finish, releases its tensor
+ * memory and returns.  Nothing waits without a limit and nothing faults; `out` is left partly
+ * or wholly unwritten.  The context stays usable: after rapid3_last_status has returned (and
+ * cleared) the code, ordinary calls compute as before.  Asynchronous on `stream`.
+ */
+int rapid3_debug_inject_timeout(rapid3_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                                int stop_group, float softmax_scale, void* stream);
 
 #ifdef __cplusplus
 }

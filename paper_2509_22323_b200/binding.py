@@ -23,6 +23,7 @@ EXPORTS = [
     "rapid3_block_scores", "rapid3_select_mask", "rapid3_sparse_joint_attn", "rapid3_gated_step",
     "rapid3_gated_step_host", "rapid3_workspace", "rapid3_launch_count", "rapid3_last_status",
     "rapid3_profile", "rapid3_profile_read", "rapid3_block_scores_static", "rapid3_static_scratch_bytes", "rapid3_cache_step", "rapid3_gated_step_device", "rapid3_gated_step_heads", "rapid3_equivalent_steps", "rapid3_select_mask_mass", "rapid3_gated_step_fused", "rapid3_gated_step_mass",
+    "rapid3_debug_inject_timeout",
 ]
 
 
@@ -69,6 +70,7 @@ def load() -> ctypes.CDLL:
     lib.rapid3_gated_step_heads.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp]
     lib.rapid3_gated_step_device.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, cf, vp]
     lib.rapid3_gated_step_host.argtypes = [vp, vp, vp, vp, vp, i32p, f32p, ci, cf, vp, i64p, i64p]
+    lib.rapid3_debug_inject_timeout.argtypes = [vp, vp, vp, vp, vp, ci, cf, vp]
     lib.rapid3_workspace.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.rapid3_launch_count.argtypes = [vp]
     lib.rapid3_launch_count.restype = ctypes.c_int64
@@ -244,6 +246,12 @@ class Context:
                                                _f32(keep_ratio), len(actions), scale, _stream(),
                                                ctypes.byref(up), ctypes.byref(down)), "rapid3_gated_step_host")
         return up.value, down.value
+
+    def rapid3_debug_inject_timeout(self, q, k, v, out, stop_group: int, softmax_scale: Optional[float] = None):
+        """Test aid: dense attention over image 0 with the failure-injection build of the kernel."""
+        scale = softmax_scale if softmax_scale is not None else self.D ** -0.5
+        _check(self.lib.rapid3_debug_inject_timeout(self.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), int(stop_group),
+                                                    scale, _stream()), "rapid3_debug_inject_timeout")
 
     # ---- helpers ----
     def workspace(self, n_sparse: int, device="cuda"):

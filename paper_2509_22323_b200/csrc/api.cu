@@ -46,7 +46,7 @@ struct rapid3_ctx {
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     std::vector<cudaEvent_t> ev_up, ev_done;                  // per image: inputs landed / output computed
     EncodeTiledFn encode = nullptr;
-    MapSlot maps[6];              // small cache keyed by base pointer
+    MapSlot maps[8];              // small cache keyed by base pointer (round-robin replacement)
     int map_rr = 0;
     int64_t launches = 0;
     // optional per-kernel timing (rapid3_profile): event pairs around each launch
@@ -98,6 +98,7 @@ int check_shape(const rapid3_shape* s) {
     if (s->block != 64) return RAPID3_ERR_UNSUPPORTED;
     if (s->D != 64 && s->D != 128) return RAPID3_ERR_UNSUPPORTED;
     if (s->B_max < 1 || s->B_max > RAPID3_MAX_IMG || s->H < 1 || s->H > 65535) return RAPID3_ERR_INVALID_ARG;
+    if ((long long)s->B_max * s->H > 65535) return RAPID3_ERR_UNSUPPORTED;     // (image, head) pairs index a grid dimension
     if (s->n_text < 0 || s->n_image < 0) return RAPID3_ERR_INVALID_ARG;
     long long N = (long long)s->n_text + s->n_image;
     if (N < 1) return RAPID3_ERR_INVALID_ARG;
@@ -121,38 +122,41 @@ int build_list(const rapid3_ctx* c, const int32_t* img_idx_host, int n_img, ImgL
 }
 
 // Tensor map over a bf16 [B, H, N, D] tensor: box = 64 channels x 64 tokens, 128-byte swizzle,
-// out-of-range tokens read as zero.
-int get_map(rapid3_ctx* c, const void* base, const CUtensorMap** out) {
+// out-of-range tokens read as zero.  The map is copied out by value at once: a later call may
+// recycle the cache slot it came from.
+int get_map(rapid3_ctx* c, const void* base, CUtensorMap* out) {
     for (auto& m : c->maps)
-        if (m.ptr == base) { *out = &m.map; return RAPID3_OK; }
+        if (m.ptr == base) { *out = m.map; return RAPID3_OK; }
     if (reinterpret_cast<uintptr_t>(base) % 16) return RAPID3_ERR_INVALID_ARG;
+    constexpr int n_slots = (int)(sizeof(c->maps) / sizeof(c->maps[0]));
     MapSlot& m = c->maps[c->map_rr];
-    c->map_rr = (c->map_rr + 1) % 6;
+    c->map_rr = (c->map_rr + 1) % n_slots;
     const rapid3_shape& s = c->shape;
     cuuint64_t dims[4] = {(cuuint64_t)s.D, (cuuint64_t)c->g.N, (cuuint64_t)s.H, (cuuint64_t)s.B_max};
     cuuint64_t strides[3] = {(cuuint64_t)s.stride_n * 2, (cuuint64_t)s.stride_h * 2, (cuuint64_t)s.stride_b * 2};
     cuuint32_t box[4] = {64, 64, 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
+    m.ptr = nullptr;
     CUresult r = c->encode(&m.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { m.ptr = nullptr; return RAPID3_ERR_CUDA; }
+    if (r != CUDA_SUCCESS) return RAPID3_ERR_CUDA;
     m.ptr = base;
-    *out = &m.map;
+    *out = m.map;
     return RAPID3_OK;
 }
 
-int attn_launch(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out, const ImgList& l,
-                const int32_t* kept_idx, const int32_t* kept_cnt, const uint64_t* bitmask, float scale,
+// `g` is the context's geometry or a copy of it narrowed to a range of heads.
+int attn_launch(rapid3_ctx* c, const TensorGeom& g, const void* q, const void* k, const void* v, void* out,
+                const ImgList& l, const int32_t* kept_idx, const int32_t* kept_cnt, const uint64_t* bitmask, float scale,
                 cudaStream_t st, const DevPlan* plan = nullptr, int n_cap = 0) {
-    const CUtensorMap *mq, *mk, *mv, *mo;
+    CUtensorMap tq, tk, tv, to;
     int r;
-    if ((r = get_map(c, q, &mq)) || (r = get_map(c, k, &mk)) || (r = get_map(c, v, &mv)) || (r = get_map(c, out, &mo)))
+    if ((r = get_map(c, q, &tq)) || (r = get_map(c, k, &tk)) || (r = get_map(c, v, &tv)) || (r = get_map(c, out, &to)))
         return r;
-    CUtensorMap tq = *mq, tk = *mk, tv = *mv, to = *mo;   // copies: a later get_map may recycle the slot
     {
         ProfScope ps(c, PROF_ATTN, st);
-        if (launch_attention(tq, tk, tv, to, c->g, l, kept_idx, kept_cnt, bitmask, scale, c->status, st, plan, n_cap) != cudaSuccess)
+        if (launch_attention(tq, tk, tv, to, g, l, kept_idx, kept_cnt, bitmask, scale, c->status, st, plan, n_cap) != cudaSuccess)
             return RAPID3_ERR_CUDA;
     }
     c->launches += 1;
@@ -202,6 +206,7 @@ int rapid3_create(rapid3_ctx** out, const rapid3_shape* shape) {
     g.n_text_blocks = (shape->n_text + 63) / 64;
     // a 128 x 128 token grid after a block-aligned text prefix: one grid row = two blocks
     // and when the text prefix is a whole number of quads, a quad is one column of four grid rows
+    g.h0 = 0;
     g.pair_stride = 1;
     if (shape->n_image == 128 * 128 && shape->n_text % 64 == 0) g.pair_stride = (g.n_text_blocks % 4 == 0) ? 3 : 2;
     g.stride_b = shape->stride_b;
@@ -343,7 +348,7 @@ int rapid3_sparse_joint_attn(rapid3_ctx* c, const void* q, const void* k, const 
     if (r != RAPID3_OK) return r;
     if (!kept_idx)
         for (int p = 0; p < n_img; ++p) l.slot[p] = -1;
-    return attn_launch(c, q, k, v, out, l, kept_idx, kept_cnt, nullptr, softmax_scale,
+    return attn_launch(c, c->g, q, k, v, out, l, kept_idx, kept_cnt, nullptr, softmax_scale,
                        static_cast<cudaStream_t>(stream));
 }
 
@@ -351,15 +356,26 @@ int rapid3_sparse_joint_attn(rapid3_ctx* c, const void* q, const void* k, const 
 // [B][H], one ratio per (image, head); an image is dense only when all its heads keep everything.
 // With `prep` set, Q and K are first produced from prep->q_raw / k_raw into q / k by the fused
 // producer, which also writes the block means: the pooling kernel is then not launched.
+// With `heads` set, only heads [heads->first, heads->first + heads->count) of the tensors are processed
+// (heads are independent; the workspace then holds that many heads, counted from 0).
+struct HeadRange {
+    int first, count;
+};
 static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,
                            const int32_t* action_host, const float* keep_ratio_host, int heads_per_ratio, int B,
                            float softmax_scale, void* stream, const PrepArgs* prep = nullptr,
-                           const float* mass_scale = nullptr) {
+                           const float* mass_scale = nullptr, const HeadRange* heads = nullptr) {
     if (!c || !q || !k || !v || !out || !action_host || !keep_ratio_host) return RAPID3_ERR_INVALID_ARG;
     if (B < 1 || B > c->shape.B_max) return RAPID3_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return RAPID3_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int n_free_img = c->g.nb - c->g.n_text_blocks - 1;
+    TensorGeom g = c->g;
+    if (heads) {
+        if (heads->first < 0 || heads->count < 1 || heads->first + heads->count > c->g.H) return RAPID3_ERR_INVALID_ARG;
+        g.h0 = heads->first;
+        g.H = heads->count;
+    }
+    const int n_free_img = g.nb - g.n_text_blocks - 1;
     // gate + compaction: sparse images (ascending batch order) get workspace slots 0..ns-1;
     // the attention list puts dense images first (longest work first), then sparse by ratio
     ImgList sparse, all;
@@ -368,7 +384,7 @@ static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const vo
     float ratio_of[RAPID3_MAX_IMG];
     // with mass_scale set, keep_ratio_host holds mass shares and the selection is the cumulative-mass rule
     const bool per_head = heads_per_ratio > 1;
-    const int H = c->g.H;
+    const int H = g.H;
     HeadKeep hk;
     MassShare share;
     if (per_head) memset(&hk, 0, sizeof hk);
@@ -418,32 +434,32 @@ static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const vo
     if (all.n == 0) return RAPID3_OK;                     // every image gated: nothing is launched
     if (prep) {
         ProfScope ps(c, PROF_POOL, st);
-        if (launch_prepare(*prep, c->g, all, sparse.n, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+        if (launch_prepare(*prep, g, all, sparse.n, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
         c->launches += 1;
     }
     if (sparse.n > 0) {
         if ((reinterpret_cast<uintptr_t>(q) % 16) || (reinterpret_cast<uintptr_t>(k) % 16)) return RAPID3_ERR_INVALID_ARG;
         if (!prep) {
             ProfScope ps(c, PROF_POOL, st);
-            if (launch_block_pool(q, k, c->g, sparse, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+            if (launch_block_pool(q, k, g, sparse, c->pooled, st) != cudaSuccess) return RAPID3_ERR_CUDA;
             c->launches += 1;
         }
         {
             ProfScope ps(c, PROF_SCORES, st);
-            if (launch_block_scores(c->pooled, c->g, sparse.n, c->scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+            if (launch_block_scores(c->pooled, g, sparse.n, c->scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
         }
         {
             ProfScope ps(c, PROF_SELECT, st);
             const cudaError_t e =
-                mass_scale ? launch_select_mask_mass(c->scores, c->g, sparse, share, *mass_scale, c->row_keep, c->bitmask,
+                mass_scale ? launch_select_mask_mass(c->scores, g, sparse, share, *mass_scale, c->row_keep, c->bitmask,
                                                      c->kept_idx, c->kept_cnt, st)
-                : per_head ? launch_select_mask_heads(c->scores, c->g, sparse, hk, c->bitmask, c->kept_idx, c->kept_cnt, st)
-                           : launch_select_mask(c->scores, c->g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st);
+                : per_head ? launch_select_mask_heads(c->scores, g, sparse, hk, c->bitmask, c->kept_idx, c->kept_cnt, st)
+                           : launch_select_mask(c->scores, g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st);
             if (e != cudaSuccess) return RAPID3_ERR_CUDA;
         }
         c->launches += mass_scale ? 3 : 2;
     }
-    return attn_launch(c, q, k, v, out, all, sparse.n ? c->kept_idx : nullptr, sparse.n ? c->kept_cnt : nullptr,
+    return attn_launch(c, g, q, k, v, out, all, sparse.n ? c->kept_idx : nullptr, sparse.n ? c->kept_cnt : nullptr,
                        sparse.n ? c->bitmask : nullptr, softmax_scale, st);
 }
 
@@ -513,7 +529,7 @@ int rapid3_gated_step_device(rapid3_ctx* c, const void* q, const void* k, const 
             return RAPID3_ERR_CUDA;
     }
     c->launches += 4;
-    return attn_launch(c, q, k, v, out, none, c->kept_idx, c->kept_cnt, c->bitmask, softmax_scale, st, c->plan, B);
+    return attn_launch(c, c->g, q, k, v, out, none, c->kept_idx, c->kept_cnt, c->bitmask, softmax_scale, st, c->plan, B);
 }
 
 int rapid3_gated_step_host(rapid3_ctx* c, const void* q_host, const void* k_host, const void* v_host, void* out_host,
@@ -576,11 +592,6 @@ int rapid3_gated_step_host(rapid3_ctx* c, const void* q_host, const void* k_host
         if (action_host[b] == RAPID3_ACT_ATTEND) last = b;
     const int H_all = s.H;
     const size_t head_bytes = (size_t)N * s.D * 2;
-    struct RestoreH {                                   // the kernels take the head count from the geometry
-        TensorGeom& g;
-        int H;
-        ~RestoreH() { g.H = H; }
-    } restore{c->g, H_all};
     for (int b = 0; b < B; ++b) {
         if (action_host[b] != RAPID3_ACT_ATTEND) continue;
         any = true;
@@ -597,14 +608,11 @@ int rapid3_gated_step_host(rapid3_ctx* c, const void* q_host, const void* k_host
             }
             if (cudaEventRecord(e_up, c->up_s) != cudaSuccess || cudaStreamWaitEvent(st, e_up, 0) != cudaSuccess)
                 return RAPID3_ERR_CUDA;
-            // heads h0 .. h0 + hn of every tensor: the same strides from a base moved by h0 heads
+            // heads h0 .. h0 + hn of image b alone: every other image is given the skip action
             one[b] = RAPID3_ACT_ATTEND;
-            c->g.H = hn;
-            const size_t hoff = h0 * head_bytes;
-            const int r = rapid3_gated_step(c, (char*)c->stage[0] + hoff, (char*)c->stage[1] + hoff,
-                                            (char*)c->stage[2] + hoff, (char*)c->stage[3] + hoff, one, keep_ratio_host, B,
-                                            softmax_scale, stream);
-            c->g.H = H_all;
+            const HeadRange hr{h0, hn};
+            const int r = gated_step_impl(c, c->stage[0], c->stage[1], c->stage[2], c->stage[3], one, keep_ratio_host, 1,
+                                          B, softmax_scale, stream, nullptr, nullptr, &hr);
             one[b] = RAPID3_ACT_SKIP;
             if (r != RAPID3_OK) return r;
             if (cudaEventRecord(e_done, st) != cudaSuccess || cudaStreamWaitEvent(c->down_s, e_done, 0) != cudaSuccess)
@@ -619,6 +627,27 @@ int rapid3_gated_step_host(rapid3_ctx* c, const void* q_host, const void* k_host
         return RAPID3_ERR_CUDA;
     if (bytes_h2d) *bytes_h2d = up;
     if (bytes_d2h) *bytes_d2h = down;
+    return RAPID3_OK;
+}
+
+int rapid3_debug_inject_timeout(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out, int stop_group,
+                                float softmax_scale, void* stream) {
+    if (!c || !q || !k || !v || !out) return RAPID3_ERR_INVALID_ARG;
+    if (stop_group < 0 || stop_group > c->g.nb) return RAPID3_ERR_INVALID_ARG;
+    if (!(softmax_scale > 0.f) || !isfinite(softmax_scale)) return RAPID3_ERR_INVALID_ARG;
+    ImgList l;
+    l.n = 1;
+    l.batch[0] = 0;
+    l.slot[0] = -1;                                       // dense: every CTA walks all nb key blocks
+    l.k_free[0] = 0;
+    CUtensorMap tq, tk, tv, to;
+    int r;
+    if ((r = get_map(c, q, &tq)) || (r = get_map(c, k, &tk)) || (r = get_map(c, v, &tv)) || (r = get_map(c, out, &to)))
+        return r;
+    if (launch_attention(tq, tk, tv, to, c->g, l, nullptr, nullptr, nullptr, softmax_scale, c->status,
+                         static_cast<cudaStream_t>(stream), nullptr, 0, stop_group) != cudaSuccess)
+        return RAPID3_ERR_CUDA;
+    c->launches += 1;
     return RAPID3_OK;
 }
 

@@ -52,8 +52,9 @@ struct MassShare {
 };
 
 struct TensorGeom {
-    int H, D, N, nb, n_text_blocks;
-    int pair_stride;                          // 1 or 2: which query blocks share an attention tile
+    int H, D, N, nb, n_text_blocks;           // H: heads this launch covers
+    int h0;                                   // first of them in the tensors (workspace arrays count heads from 0)
+    int pair_stride;                          // 1, 2 or 3: which query blocks share an attention tile
     long long stride_b, stride_h, stride_n;   // elements
 };
 
@@ -95,9 +96,10 @@ cudaError_t launch_prepare(const PrepArgs& a, const TensorGeom& g, const ImgList
 cudaError_t launch_plan(const int32_t* action_dev, const float* ratio_dev, int B, const TensorGeom& g,
                         DevPlan* plan, int* status, cudaStream_t s);
 // K3: attention over kept tiles.  `bitmask` (optional) is the select kernel's bitmask of the same
-// lists; when present the kernel reads it instead of walking the lists.
+// lists; when present the kernel reads it instead of walking the lists.  inject_stop_group >= 0
+// launches the failure-injection build of the kernel (see rapid3_debug_inject_timeout).
 cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv,
                              const CUtensorMap& tmo, const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
                              const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* status,
-                             cudaStream_t s, const DevPlan* plan = nullptr, int n_cap = 0);
+                             cudaStream_t s, const DevPlan* plan = nullptr, int n_cap = 0, int inject_stop_group = -1);
 cudaError_t attention_static_init();

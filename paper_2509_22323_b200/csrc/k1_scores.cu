@@ -28,7 +28,7 @@ __global__ void __launch_bounds__(128) pool_kernel(const uint16_t* __restrict__ 
     const int p = blockIdx.z - which * n_cap;
     if (plan && p >= plan->sparse.n) return;          // device-resident plan: fewer images than the grid covers
     const int batch = plan ? plan->sparse.batch[p] : imgs.batch[p];
-    const uint16_t* base = (which ? k : q) + (long long)batch * g.stride_b + (long long)h * g.stride_h;
+    const uint16_t* base = (which ? k : q) + (long long)batch * g.stride_b + (long long)(g.h0 + h) * g.stride_h;
     const int c = lane % TPR, r0 = lane / TPR;
     const int n0 = blk * 64;
     const int valid = min(64, g.N - n0);
@@ -206,6 +206,7 @@ extern "C" int rapid3_block_scores_static(const rapid3_shape* s, const void* q, 
     if (!s || !q || !k || !scores) return RAPID3_ERR_INVALID_ARG;
     if (s->block != RAPID3_BLOCK || (s->D != 64 && s->D != 128)) return RAPID3_ERR_UNSUPPORTED;
     if (s->B_max < 1 || s->B_max > RAPID3_MAX_IMG || s->H < 1 || s->H > 65535) return RAPID3_ERR_INVALID_ARG;
+    if ((long long)s->B_max * s->H > 65535) return RAPID3_ERR_UNSUPPORTED;     // (image, head) pairs index a grid dimension
     if (s->n_text < 0 || s->n_image < 0) return RAPID3_ERR_INVALID_ARG;
     const long long N = (long long)s->n_text + s->n_image;
     if (N < 1) return RAPID3_ERR_INVALID_ARG;
@@ -221,6 +222,7 @@ extern "C" int rapid3_block_scores_static(const rapid3_shape* s, const void* q, 
     g.N = (int)N;
     g.nb = (int)((N + 63) / 64);
     g.n_text_blocks = (s->n_text + 63) / 64;
+    g.h0 = 0;
     g.pair_stride = 1;
     g.stride_b = s->stride_b;
     g.stride_h = s->stride_h;

@@ -51,6 +51,7 @@ struct AttnParams {
     const DevPlan* plan;           // optional: image list and n_dense from device memory (grid sized for n_cap images)
     int* status;
     float scale_log2;
+    int stop_group;                // failure-injection build of the kernel only: the producer stops before this group
 };
 
 template <int D>
@@ -86,7 +87,11 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
-template <int D>
+// INJECT = true is the failure-injection build behind rapid3_debug_inject_timeout: the producer
+// stops before group prm.stop_group and every wait gives up after 2^12 polls, so the waits of all
+// roles run out and the abort path (status word, drain of the copies in flight, UMMA drain, TMEM
+// release) is what runs.  The product launches only use INJECT = false.
+template <int D, bool INJECT = false>
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
             const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo, const AttnParams prm) {
@@ -201,7 +206,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             for (int dh = 0; dh < DH; ++dh)
                 tma_load_4d(sQ + (ps2 ? (a & 1) : (a >> 1)) * C::QTILE_BYTES + dh * QHALF_BYTES +
                                 (ps2 ? (a >> 1) : (a & 1)) * BLK_BYTES, &tmq, bQ,
-                            dh * 64, qblk(a) * 64, h, b);
+                            dh * 64, qblk(a) * 64, g.h0 + h, b);
     }
 
     // ---------------------------------------------------------------- union of the four kept lists
@@ -261,7 +266,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     };
     // bounded wait that also gives up quickly once another role has failed
     auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
-        for (uint32_t it = 0; it < (1u << 22); ++it) {
+        constexpr uint32_t limit = INJECT ? (1u << 12) : (1u << 22);
+        for (uint32_t it = 0; it < limit; ++it) {
             if (mbar_try_wait(bar, parity)) return true;
             if ((it & 255u) == 255u && ctl->abort_flag) return false;
         }
@@ -294,20 +300,23 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                     const int blk = ctl->u_blk[gi];
 #pragma unroll
                     for (int dh = 0; dh < DH; ++dh)
-                        tma_load_4d(sK + s * C::KV_BYTES + dh * BLK_BYTES, &tmk, bKF + 8 * s, dh * 64, blk * 64, h, b);
+                        tma_load_4d(sK + s * C::KV_BYTES + dh * BLK_BYTES, &tmk, bKF + 8 * s, dh * 64, blk * 64, g.h0 + h, b);
                 }
                 if (has_v) {
                     const int blk = ctl->u_blk[jv];
 #pragma unroll
                     for (int dh = 0; dh < DH; ++dh)
-                        tma_load_4d(sV + sv * C::KV_BYTES + dh * BLK_BYTES, &tmv, bKF + 8 * s, dh * 64, blk * 64, h, b);
+                        tma_load_4d(sV + sv * C::KV_BYTES + dh * BLK_BYTES, &tmv, bKF + 8 * s, dh * 64, blk * 64, g.h0 + h, b);
                 }
                 g_issued = gi + 1;
                 return true;
             };
             bool ok = true;
-            for (int gi = 0; ok && n_u > 0 && gi <= n_u; ++gi) ok = load_group(gi);
-            if (ctl->abort_flag) {
+            for (int gi = 0; ok && n_u > 0 && gi <= n_u; ++gi) {
+                if (INJECT && gi == prm.stop_group) break;
+                ok = load_group(gi);
+            }
+            if (INJECT || ctl->abort_flag) {
                 // drain: do not leave the CTA while bulk copies may still land in its shared memory
                 mbar_wait(bQ, 0, 1u << 20);
                 for (int gi = max(0, g_issued - KS); gi < g_issued; ++gi)
@@ -540,7 +549,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
 #pragma unroll
             for (int dh = 0; dh < DH; ++dh)
                 tma_store_4d(&tmo, sQ + t * C::QTILE_BYTES + dh * QHALF_BYTES + (wl >> 1) * BLK_BYTES, dh * 64,
-                             qblk(qb_id) * 64, h, b);
+                             qblk(qb_id) * 64, g.h0 + h, b);
             bulk_commit_group();
             bulk_wait_read_all();
         }
@@ -577,6 +586,12 @@ cudaError_t attention_static_init() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem_bytes<64>());
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_smem_bytes<128>());
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)attn_smem_bytes<64>());
+    if (e != cudaSuccess) return e;
     g_attr_set = true;
     return cudaSuccess;
 }
@@ -585,7 +600,7 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
                              const CUtensorMap& tmo,
                              const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
                              const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* status,
-                             cudaStream_t s, const DevPlan* plan, int n_cap) {
+                             cudaStream_t s, const DevPlan* plan, int n_cap, int inject_stop_group) {
     if (!g_attr_set) {
         cudaError_t e = attention_static_init();
         if (e != cudaSuccess) return e;
@@ -603,10 +618,17 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
     while (n_dense < imgs.n && (imgs.slot[n_dense] < 0 || kept_idx == nullptr)) ++n_dense;
     prm.n_dense = n_dense;
     prm.plan = plan;
+    prm.stop_group = inject_stop_group;
     dim3 grid(((g.nb + 3) / 4) * g.H * (plan ? n_cap : imgs.n), 1, 1);
-    if (g.D == 128)
+    if (inject_stop_group >= 0) {
+        if (g.D == 128)
+            attn_kernel<128, true><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, tmo, prm);
+        else
+            attn_kernel<64, true><<<grid, NTHREADS, attn_smem_bytes<64>(), s>>>(tmq, tmk, tmv, tmo, prm);
+    } else if (g.D == 128) {
         attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, tmo, prm);
-    else
+    } else {
         attn_kernel<64><<<grid, NTHREADS, attn_smem_bytes<64>(), s>>>(tmq, tmk, tmv, tmo, prm);
+    }
     return cudaGetLastError();
 }

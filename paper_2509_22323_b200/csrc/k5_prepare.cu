@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(128, PREP_MINB) prepare_kernel(const uint16_t*
     const int which = blockIdx.z / imgs.n;            // 0 = Q, 1 = K
     const int p = blockIdx.z - which * imgs.n;
     const int batch = imgs.batch[p], slot = imgs.slot[p];
-    const long long off = (long long)batch * g.stride_b + (long long)h * g.stride_h;
+    const long long off = (long long)batch * g.stride_b + (long long)(g.h0 + h) * g.stride_h;
     const uint16_t* src = (which ? k_raw : q_raw) + off;
     uint16_t* dst = (which ? k_out : q_out) + off;
     const float* gain = which ? k_gain : q_gain;

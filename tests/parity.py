@@ -16,12 +16,13 @@ TIE_EPS = 1e-6
 
 def compare_masks(gpu_mask: np.ndarray, ora_mask: np.ndarray, gap: np.ndarray, what: str = ""):
     """gpu_mask, ora_mask: [H, nb, nb] uint8; gap: [H, nb].  Rows whose last-kept / first-dropped
-    scores lie within 1e-6 are near ties: a flip there is reported, every other row must match
-    bit for bit.  Returns the list of flipped near-tie rows."""
+    scores differ by more than 0 and at most 1e-6 are near ties: a flip there is reported, every
+    other row must match bit for bit -- including rows with gap exactly 0, where the scores are
+    equal and the lower block index decides.  Returns the list of flipped near-tie rows."""
     diff_rows = np.argwhere((gpu_mask != ora_mask).any(axis=-1))
     flips = []
     for h, i in diff_rows:
-        if gap[h, i] <= TIE_EPS:
+        if 0.0 < gap[h, i] <= TIE_EPS:
             flips.append((int(h), int(i), float(gap[h, i])))
         else:
             raise AssertionError(f"{what}: mask row (head {h}, block {i}) differs, gap {gap[h, i]:.3e}\n"
@@ -78,17 +79,44 @@ def compare_outputs(gpu_out: torch.Tensor, ora_out: np.ndarray, what: str = "", 
     return mx, mean
 
 
-def oracle_image(q, k, v, n_text, ratio, scale, heads, qblocks):
-    """Oracle scores/mask on all heads, attention only on the sampled heads x query blocks."""
-    S32, mask, gap = oracle.image_mask(q, k, n_text, ratio)
-    return S32, mask, gap
+def bf16_bits(t: torch.Tensor) -> np.ndarray:
+    """bf16 tensor -> uint16 numpy array of its bit patterns (one copy to the host)."""
+    return np.ascontiguousarray(t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16))
 
 
 def oracle_out_samples(q, k, v, mask, scale, heads, qblocks):
-    H, N, D = q.shape
+    """Oracle attention on the (head, query block) units heads x qblocks; NaN elsewhere."""
+    return oracle_out_units(q, k, v, mask, scale, [(h, i) for h in heads for i in qblocks])
+
+
+def oracle_out_units(q, k, v, mask, scale, units):
+    """Oracle attention of one image on a list of (head, query block) units, each computed by one
+    call of the oracle on that head alone; rows of every other unit stay NaN.  q, k, v: bf16
+    [H, N, D] tensors (converted to bit patterns once)."""
+    qb, kb, vb = bf16_bits(q), bf16_bits(k), bf16_bits(v)
+    H, N, D = qb.shape
     out = np.full((H, N, D), np.nan)
-    for h in heads:
-        for i in qblocks:
-            part = oracle.masked_attention(q, k, v, mask, scale, qb_lo=i, qb_hi=i + 1, heads=[h])
-            out[h, 64 * i:64 * i + 64] = part[h, 64 * i:64 * i + 64]
+    for h, i in units:
+        part = oracle.masked_attention(qb[h:h + 1], kb[h:h + 1], vb[h:h + 1], mask[h:h + 1], scale, qb_lo=i, qb_hi=i + 1)
+        out[h, 64 * i:64 * i + 64] = part[0, 64 * i:64 * i + 64]
     return out
+
+
+def sample_units(n_heads: int, nb: int, ntb: int, count: int, seed: int):
+    """Seeded sample of (head, query block) units of one image: per head the first and last text
+    block, the first image block and the last two blocks (the tail), then uniformly drawn units up
+    to `count`.  Every head and every position of a block within its quad of four is covered."""
+    rng = np.random.default_rng(seed)
+    units = set()
+    for h in range(n_heads):
+        for i in (0, ntb - 1, ntb, nb - 2, nb - 1):
+            if 0 <= i < nb and (h + i) % 3 == 0:
+                units.add((h, i))
+        units.add((h, int(rng.integers(0, nb))))
+    while len(units) < min(count, n_heads * nb):
+        units.add((int(rng.integers(0, n_heads)), int(rng.integers(0, nb))))
+    units = sorted(units)
+    assert {h for h, _ in units} == set(range(n_heads))
+    if nb >= 8 and count >= 64:
+        assert {i % 4 for _, i in units} == {0, 1, 2, 3} and {(i // 2) % 2 for _, i in units} == {0, 1}
+    return units

@@ -34,6 +34,11 @@ def test_strerror_and_shape_helpers_run_on_the_host():
     assert lib.rapid3_num_blocks(ctypes.byref(s2)) == 70
     bad = binding.Shape(1, 2, 96, 64, 256, 64, 1, 1, 96)
     assert lib.rapid3_num_blocks(ctypes.byref(bad)) == -2
+    # (image, head) pairs index one grid dimension: more than 65535 of them is an unsupported shape
+    wide = binding.Shape(64, 2048, 64, 64, 256, 64, 2048 * 320 * 64, 320 * 64, 64)
+    assert lib.rapid3_num_blocks(ctypes.byref(wide)) == -2
+    handle = ctypes.c_void_p()
+    assert lib.rapid3_create(ctypes.byref(handle), ctypes.byref(wide)) == -2 and not handle.value
 
 
 def test_null_context_is_refused_before_any_gpu_call():
@@ -55,6 +60,7 @@ def test_null_context_is_refused_before_any_gpu_call():
     assert lib.rapid3_gated_step_fused(null, null, null, null, null, null, null, 1e-6, null, null, null, one_i, one_f, 1,
                                        1.0, null) == -1
     assert lib.rapid3_gated_step_host(null, null, null, null, null, one_i, one_f, 1, 1.0, null, null, null) == -1
+    assert lib.rapid3_debug_inject_timeout(null, null, null, null, null, 0, 1.0, null) == -1
     assert lib.rapid3_profile(null, 1) == -1
     assert lib.rapid3_launch_count(null) == -1
     assert lib.rapid3_destroy(null) in (0, -1)

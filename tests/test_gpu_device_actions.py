@@ -1,10 +1,14 @@
-"""rapid3_gated_step_device: policy actions and keep ratios stay on the GPU.  Output and
-workspace must equal those of rapid3_gated_step given the same decisions from the host."""
+"""rapid3_gated_step_device: policy actions and keep ratios stay on the GPU.  Masks and outputs
+are checked against the oracle's gated step (Sec. 3.3: the heads sample their actions on the
+device; the step they gate is the same one), and must also equal those of rapid3_gated_step
+given the same decisions from the host."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2509_22323_b200 import binding, inputs
+from tests import parity
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -42,6 +46,19 @@ def test_device_actions_equal_host_actions(case):
     for b, a in enumerate(acts):
         if a != 2:
             assert (out_d[b].view(torch.int16) == np.int16(POISON)).all()
+    # against the oracle: masks of the sparse images (slots in ascending batch order), outputs of all attending ones
+    ref = oracle.gated_step(Q.cpu(), K.cpu(), V.cpu(), acts, ratios, wl.n_text, wl.softmax_scale)
+    sparse = [b for b, (a, r) in enumerate(zip(acts, ratios)) if a == 2 and r < 1.0]
+    if sparse:
+        ws = ctx_d.workspace(len(sparse))
+        dense = binding.bitmask_to_dense(ws[1], wl.n_blocks).numpy()
+        parity.check_lists(ws[2], ws[3], dense)
+        for slot, b in enumerate(sparse):
+            parity.compare_masks(dense[slot], ref[b]["mask"], ref[b]["gap"], f"device actions {name} img {b}")
+    for b, a in enumerate(acts):
+        if a == 2:
+            assert not (out_d[b].view(torch.int16) == np.int16(POISON)).any()
+            parity.compare_outputs(out_d[b], ref[b]["out"], f"device actions {name} img {b} ratio {ratios[b]}")
 
 
 def test_device_actions_flag_invalid_decisions():
@@ -87,3 +104,9 @@ def test_device_actions_change_between_graph_replays():
         ctx_h.rapid3_gated_step(Q, K, V, want, acts, ratios, wl.softmax_scale)
         torch.cuda.synchronize()
         assert torch.equal(out.view(torch.int16), want.view(torch.int16)), (acts, ratios)
+        ref = oracle.gated_step(Q.cpu(), K.cpu(), V.cpu(), acts, ratios, wl.n_text, wl.softmax_scale)
+        for b, a in enumerate(acts):
+            if a == 2:
+                parity.compare_outputs(out[b], ref[b]["out"], f"graph replay {acts} img {b}")
+            else:
+                assert (out[b].view(torch.int16) == np.int16(POISON)).all()
