@@ -242,15 +242,20 @@ class Prepared:
         from paper_2509_22323_b200 import binding
         self.binding, self.wl, self.dev = binding, wl, dev
         self.ctx = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
-        nsets = 2
+        self.set_bytes = 3 * wl.batch * wl.heads * wl.n_tokens * wl.head_dim * 2
+        # input sets are rotated so that a step never finds its inputs in L2 (126 MB): enough sets that the
+        # others together exceed 200 MB; the `tiny` workload would need hundreds, so there a buffer larger
+        # than L2 is rewritten before every step instead (outside the step's event pair)
+        nsets = max(2, -(-200_000_000 // self.set_bytes) + 1)
+        self.flush = None
+        if nsets > 8:
+            nsets = 2
+            self.flush = torch.empty(192 << 20, dtype=torch.uint8, device=dev)
         steps_of = list(range(nsets))
         if wl.steps > 1:
             steps_of = list(range(wl.steps))           # the gated trajectory: fresh Q/K/V per step
             nsets = min(wl.steps, 4)
         self.nsets = nsets
-        # inputs larger than L2 are rotated; small ones (the `tiny` workload) need an explicit flush
-        self.set_bytes = 3 * wl.batch * wl.heads * wl.n_tokens * wl.head_dim * 2
-        self.flush = torch.empty(192 << 20, dtype=torch.uint8, device=dev) if self.set_bytes * nsets < (160 << 20) else None
         # each rank draws its own data (weak scaling): shift the step index by the rank
         self.sets = [inputs.make_qkv(wl, rank_step(rank, st), device=dev) for st in range(nsets)]
         self.out = torch.empty_like(self.sets[0][0])
@@ -275,8 +280,6 @@ class Prepared:
 
     def step(self, i):
         (Q, K, V), acts, ratios = self.plan[i % len(self.plan)]
-        if self.flush is not None:
-            self.flush.fill_(i & 0xFF)                 # evicts the small inputs from L2 between steps
         self.ctx.rapid3_gated_step(Q, K, V, self.out, acts, ratios, self.wl.softmax_scale)
 
     def flops(self, steps):
@@ -284,7 +287,8 @@ class Prepared:
 
     def l2_note(self):
         if self.flush is not None:
-            return f"inputs smaller than L2: a {self.flush.numel() >> 20} MiB buffer is rewritten between steps"
+            return (f"inputs smaller than L2: a {self.flush.numel() >> 20} MiB buffer is rewritten before every step, "
+                    "each step between its own event pair")
         return f"inputs larger than L2 ({self.set_bytes / 1e6:.0f} MB per set), {self.nsets} input sets rotated"
 
 
@@ -302,17 +306,20 @@ def timed_region(pw, steps, warmup, dist=None):
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     w0 = time.time()
-    e0.record()
-    for i in range(steps):
-        pw.step(i)
-    e1.record()
-    torch.cuda.synchronize()
+    if pw.flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            pw.step(i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_total = e0.elapsed_time(e1)
+    else:
+        ms_total = sum(per_step_times(pw, steps))   # L2 flushed before every step, outside its event pair
     w1 = time.time()
     if dist is not None:
         dist.barrier()
-    ms_total = e0.elapsed_time(e1)
     launches = ctx.launch_count() - n0
     attn = ctx.profile_read()["attention"]
     ctx.profile(False)
@@ -320,23 +327,18 @@ def timed_region(pw, steps, warmup, dist=None):
 
 
 def per_step_times(pw, n):
-    """n further steps, each between its own event pair: median and minimum of the step time."""
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    """n steps, each between its own event pair (for a workload smaller than L2 the flush buffer is
+    rewritten before the pair): the list of step times in ms."""
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
     torch.cuda.synchronize()
-    for i in range(n):
+    for i, (a, b) in enumerate(pairs):
         if pw.flush is not None:
             pw.flush.fill_(i & 0xFF)
-        (Q, K, V), acts, ratios = pw.plan[i % len(pw.plan)]
-        evs[i].record()
-        pw.ctx.rapid3_gated_step(Q, K, V, pw.out, acts, ratios, pw.wl.softmax_scale)
-        evs[i + 1].record() if i == n - 1 else None
+        a.record()
+        pw.step(i)
+        b.record()
     torch.cuda.synchronize()
-    # step i runs from its own record to the next step's record (the flush of a small workload sits before the record)
-    if pw.flush is None:
-        ts = [evs[i].elapsed_time(evs[i + 1]) for i in range(n)]
-    else:
-        ts = None
-    return ts
+    return [a.elapsed_time(b) for a, b in pairs]
 
 
 def side_kernels(pw, n):
