@@ -8,18 +8,18 @@
 // kept; inside a tile a 64x64 sub-tile whose key block is not in that query block's own list
 // gets P = 0, so each query block attends exactly its own kept set.
 //
-// Roles (352 threads):
-//   warp 8      producer: TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of Q once, then
+// Roles (608 threads):
+//   warp 16     producer: TMA loads (cp.async.bulk.tensor, 128-byte swizzle) of Q once, then
 //               the gathered K and V blocks into two rings of shared-memory stages; K(g) and
 //               V(g - 1), which the MMA warps need together, complete one barrier
-//   warps 9,10  UMMA issue, one warp per tile (warp 9 also owns the TMEM allocation).  S of a
+//   warps 17,18 UMMA issue, one warp per tile (warp 17 also owns the TMEM allocation).  S of a
 //               tile is double buffered in TMEM (2 x 64 fp32 columns): S(n+1) = Q K^T is issued
 //               before O += P(n) V, so the tensor pipe works on the next scores while the
 //               softmax warps are busy with the current ones.  Both warps walk the same union
 //               list one block ahead in K than in V; a stage is released when both have passed it
-//   warps 0-7   softmax, four warps per tile: thread = one query row; S(n) from TMEM in one pass
-//               (64 registers), fp32 online softmax with lazy rescale of O, P(n) written back
-//               over S(n) as bf16, final O / l store
+//   warps 0-15  softmax, eight warps per tile and four per SM sub-partition: a warp owns 16 query rows, a
+//               thread a quarter of two rows (16x256b fragments; 32 scores per key block); fp32 online
+//               softmax with lazy rescale of O, P(n) written back over S(n) as bf16, final O / l store
 // TMEM: tile t owns columns [256 t, 256 t + 256): S(n) at 64 (n & 1), O at 128.
 // Every mbarrier wait is bounded; a wait that runs out records RAPID3_ERR_TIMEOUT in the status
 // word and the CTA drains its copies, releases its TMEM and exits normally.
@@ -30,8 +30,9 @@ using namespace ptx;
 
 namespace {
 
-constexpr int NTHREADS = 352;
-constexpr int PRODUCER_WARP = 8, MMA_WARP0 = 9;
+constexpr int SOFTMAX_WARPS = 16;
+constexpr int PRODUCER_WARP = 16, MMA_WARP0 = 17;
+constexpr int NTHREADS = 32 * (SOFTMAX_WARPS + 3);
 constexpr int TMEM_COLS = 512;
 constexpr int TILE_COLS = 256;      // TMEM columns of one Q tile
 constexpr int O_COL = 128;
@@ -174,7 +175,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         }
         for (int s = 0; s < 4; ++s) {
             mbar_init(bSF + 8 * s, 1);
-            mbar_init(bPF + 8 * s, 4);      // one arrival per softmax warp of the tile
+            mbar_init(bPF + 8 * s, 8);      // one arrival per softmax warp of the tile
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(bPV + 8 * t, 1);
@@ -399,19 +400,26 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         __syncwarp();
     } else {
         // ------------------------------------------------------------ softmax / correction / epilogue
-        const int t = warp >> 2, wl = warp & 3;        // tile, lane quarter of the tile
+        // Sixteen warps, four per SM sub-partition, so that while one waits on a barrier or on tensor memory
+        // the others keep the exponential unit busy.  Warp w works on tile (w >> 2) & 1, on the 16 rows
+        // 32 (w & 3) + 16 (w >> 3) .. + 15 of it, with the 16x256b fragment layout: a thread owns two rows
+        // (r_lo = lane / 4 and r_lo + 8 of the sixteen) and, of every group of eight score columns, the pair
+        // 2 (lane % 4), + 1 -- 32 scores per key block.  The four threads of a quad share their rows' maximum
+        // with two shuffles, and only when some row of the warp may have grown.
+        const int t = (warp >> 2) & 1, wl = warp & 3, hf = warp >> 3;
         const int a = ps2 ? 2 * (wl >> 1) + t : 2 * t + (wl >> 1);   // query block of the quad
         const uint32_t tile_bits = ps2 ? (5u << t) : (3u << (2 * t));
-        const int row = wl * 32 + lane;                // row of the 128-row tile == TMEM lane
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(wl * 32) << 16) + t * TILE_COLS;
+        const int cg = lane & 3;                        // column pair within a group of eight
+        const int row_lo = wl * 32 + hf * 16 + (lane >> 2);          // row of the 128-row tile; the second row is + 8
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(wl * 32 + hf * 16) << 16) + t * TILE_COLS;
         const uint32_t tO = lane_addr + O_COL;
         const uint32_t bSFt = bSF + 16 * t, bPFt = bPF + 16 * t, bPVt = bPV + 8 * t;
         const float c2 = prm.scale_log2;
         const int tail_valid = N - (nb - 1) * 64;      // valid tokens of the last block (1..64)
-        float m_run = -INFINITY;
-        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+        float m_lo = -INFINITY, m_hi = -INFINITY;      // reference maxima of the two rows
+        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;  // partial row sums: (l0, l1) first row, (l2, l3) second row
         bool ok = true;
-        uint32_t r0[32], r1[32];
+        uint32_t r[32];
         int n = 0;                                     // blocks of this tile so far
         for (int j = 0; j < n_u; ++j) {
             const uint32_t f = ctl->u_flag[j];
@@ -423,88 +431,82 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             const uint32_t tS = lane_addr + 64 * buf;
             if (!(ok = wait_warp(bSFt + 8 * buf, (n >> 1) & 1))) break;
             tc_fence_after();
+            uint32_t pk[16];
             if (act) {
-                tmem_ld32(tS, r0);
-                tmem_ld32(tS + 32, r1);
+                tmem_ld16x256_x8(tS, r);
                 tc_wait_ld();
                 if (valid != 64) {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        if (e >= valid) r0[e] = 0xff800000u;          // -inf: outside the sequence
-                        if (32 + e >= valid) r1[e] = 0xff800000u;
-                    }
+                    for (int k = 0; k < 8; ++k)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e)
+                            if (8 * k + 2 * cg + e >= valid) {       // -inf: outside the sequence
+                                r[4 * k + e] = 0xff800000u;
+                                r[4 * k + 2 + e] = 0xff800000u;
+                            }
                 }
-                // One pass over the 64 scores gives P = 2^(S c2 - m c2) (packed to bf16), the block's
-                // partial row sums and the block's row maximum.  The pass runs with the reference
-                // maximum m as it stands, so the exponentials do not wait for this block's maximum;
-                // only when a row's maximum has grown by more than 2^8 (rare after the first blocks,
-                // always at the first block) O and l are rescaled and the pass is repeated.
-                uint32_t pk[32];
+                // One pass over the 32 scores gives P = 2^(S c2 - m c2) (packed to bf16), the block's partial
+                // row sums and the thread's share of the block's row maxima.  The pass runs with the reference
+                // maxima as they stand, so the exponentials do not wait for this block's maximum; only when a
+                // row's maximum has grown by more than 2^8 (rare after the first blocks, always at the first
+                // block) O and l are rescaled and the pass is repeated.
                 float b0, b1, b2, b3;
                 bool redo;
                 do {
-                    const float ms = m_run * c2;
-                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                    const float ms_lo = m_lo * c2, ms_hi = m_hi * c2;
+                    float mx_lo = -INFINITY, mx_hi = -INFINITY;
                     b0 = b1 = b2 = b3 = 0.f;
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
+                    for (int k = 0; k < 8; ++k) {
                         float x0, x1, x2, x3;
-                        fma2(x0, x1, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]), c2, -ms);
-                        fma2(x2, x3, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]), c2, -ms);
+                        fma2(x0, x1, __uint_as_float(r[4 * k]), __uint_as_float(r[4 * k + 1]), c2, -ms_lo);
+                        fma2(x2, x3, __uint_as_float(r[4 * k + 2]), __uint_as_float(r[4 * k + 3]), c2, -ms_hi);
                         x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
                         add2(b0, b1, x0, x1);
                         add2(b2, b3, x2, x3);
-                        pk[e / 2] = pack_bf16(x0, x1);
-                        pk[e / 2 + 1] = pack_bf16(x2, x3);
-                        mx0 = max3(mx0, __uint_as_float(r0[e]), __uint_as_float(r0[e + 1]));
-                        mx1 = max3(mx1, __uint_as_float(r0[e + 2]), __uint_as_float(r0[e + 3]));
+                        pk[2 * k] = pack_bf16(x0, x1);
+                        pk[2 * k + 1] = pack_bf16(x2, x3);
+                        mx_lo = max3(mx_lo, __uint_as_float(r[4 * k]), __uint_as_float(r[4 * k + 1]));
+                        mx_hi = max3(mx_hi, __uint_as_float(r[4 * k + 2]), __uint_as_float(r[4 * k + 3]));
                     }
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        float x0, x1, x2, x3;
-                        fma2(x0, x1, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]), c2, -ms);
-                        fma2(x2, x3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]), c2, -ms);
-                        x0 = ex2(x0); x1 = ex2(x1); x2 = ex2(x2); x3 = ex2(x3);
-                        add2(b0, b1, x0, x1);
-                        add2(b2, b3, x2, x3);
-                        pk[16 + e / 2] = pack_bf16(x0, x1);
-                        pk[16 + e / 2 + 1] = pack_bf16(x2, x3);
-                        mx2 = max3(mx2, __uint_as_float(r1[e]), __uint_as_float(r1[e + 1]));
-                        mx3 = max3(mx3, __uint_as_float(r1[e + 2]), __uint_as_float(r1[e + 3]));
-                    }
-                    const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-                    const bool grow = (mx - m_run) * c2 > RESCALE_LOG2;       // true from -inf
-                    redo = __any_sync(0xffffffffu, grow);
+                    // a thread sees a quarter of each row: if any thread of the warp sees growth, the quads
+                    // combine their maxima and decide row by row
+                    redo = __any_sync(0xffffffffu, (mx_lo - m_lo) * c2 > RESCALE_LOG2 || (mx_hi - m_hi) * c2 > RESCALE_LOG2);
                     if (redo) {
-                        const bool fix_o = grow && m_run != -INFINITY;        // O holds something to rescale
-                        if (__any_sync(0xffffffffu, fix_o)) {
+                        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+                        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+                        mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+                        mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+                        const bool g_lo = (mx_lo - m_lo) * c2 > RESCALE_LOG2, g_hi = (mx_hi - m_hi) * c2 > RESCALE_LOG2;   // true from -inf
+                        const bool f_lo = g_lo && m_lo != -INFINITY, f_hi = g_hi && m_hi != -INFINITY;   // O holds something to rescale
+                        if (__any_sync(0xffffffffu, f_lo || f_hi)) {
                             // O must be at rest: wait for P(n-1) V
                             if (!(ok = wait_warp(bPVt, (n - 1) & 1))) break;
                             tc_fence_after();
-                            const float alpha = fix_o ? ex2((m_run - mx) * c2) : 1.f;
-                            l0 *= alpha; l1 *= alpha; l2 *= alpha; l3 *= alpha;
-                            uint32_t o[32];
+                            const float a_lo = f_lo ? ex2((m_lo - mx_lo) * c2) : 1.f, a_hi = f_hi ? ex2((m_hi - mx_hi) * c2) : 1.f;
+                            l0 *= a_lo; l1 *= a_lo; l2 *= a_hi; l3 *= a_hi;
+                            uint32_t o[16];
 #pragma unroll
                             for (int ch = 0; ch < D / 32; ++ch) {
-                                tmem_ld32(tO + ch * 32, o);
+                                tmem_ld16x256_x4(tO + ch * 32, o);
                                 tc_wait_ld();
 #pragma unroll
-                                for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                                tmem_st32(tO + ch * 32, o);
+                                for (int e = 0; e < 16; ++e)
+                                    o[e] = __float_as_uint(__uint_as_float(o[e]) * ((e & 2) ? a_hi : a_lo));
+                                tmem_st16x256_x4(tO + ch * 32, o);
                             }
                         }
-                        if (grow) m_run = mx;
+                        if (g_lo) m_lo = mx_lo;
+                        if (g_hi) m_hi = mx_hi;
                     }
                 } while (redo);
                 if (!ok) break;
                 l0 += b0; l1 += b1; l2 += b2; l3 += b3;
-                tmem_st32(tS, pk);
             } else {
-                uint32_t z[32];
 #pragma unroll
-                for (int e = 0; e < 32; ++e) z[e] = 0u;
-                tmem_st32(tS, z);
+                for (int e = 0; e < 16; ++e) pk[e] = 0u;
             }
+            tmem_st16x128_x8(tS, pk);
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
@@ -517,35 +519,41 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         if (ok && n > 0) ok = wait_warp(bOD + 8 * t, 0);
         if (ok) {
             tc_fence_after();
-            const float l_run = (l0 + l1) + (l2 + l3);
-            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            uint8_t* so = smem + t * C::QTILE_BYTES + row * 128;
+            float s_lo = l0 + l1, s_hi = l2 + l3;      // the quad's four partial sums make the row sum
+            s_lo += __shfl_xor_sync(0xffffffffu, s_lo, 1);
+            s_hi += __shfl_xor_sync(0xffffffffu, s_hi, 1);
+            s_lo += __shfl_xor_sync(0xffffffffu, s_lo, 2);
+            s_hi += __shfl_xor_sync(0xffffffffu, s_hi, 2);
+            const float inv_lo = s_lo > 0.f ? 1.f / s_lo : 0.f, inv_hi = s_hi > 0.f ? 1.f / s_hi : 0.f;
+            uint8_t* so_lo = smem + t * C::QTILE_BYTES + row_lo * 128;
+            uint8_t* so_hi = so_lo + 8 * 128;
+            const int sw_lo = row_lo & 7, sw_hi = (row_lo + 8) & 7;
+            uint32_t o[16];
 #pragma unroll
             for (int ch = 0; ch < D / 32; ++ch) {
                 if (n > 0) {
-                    tmem_ld32(tO + ch * 32, r0);
+                    tmem_ld16x256_x4(tO + ch * 32, o);
                     tc_wait_ld();
                 } else {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) r0[e] = 0u;
+                    for (int e = 0; e < 16; ++e) o[e] = 0u;
                 }
 #pragma unroll
-                for (int v4 = 0; v4 < 4; ++v4) {
-                    uint4 o;
-                    o.x = pack_bf16(__uint_as_float(r0[v4 * 8 + 0]) * inv, __uint_as_float(r0[v4 * 8 + 1]) * inv);
-                    o.y = pack_bf16(__uint_as_float(r0[v4 * 8 + 2]) * inv, __uint_as_float(r0[v4 * 8 + 3]) * inv);
-                    o.z = pack_bf16(__uint_as_float(r0[v4 * 8 + 4]) * inv, __uint_as_float(r0[v4 * 8 + 5]) * inv);
-                    o.w = pack_bf16(__uint_as_float(r0[v4 * 8 + 6]) * inv, __uint_as_float(r0[v4 * 8 + 7]) * inv);
-                    const int chunk = (ch & 1) * 4 + v4;            // 16-byte chunk of the 128-byte half row
-                    *reinterpret_cast<uint4*>(so + (ch >> 1) * QHALF_BYTES + ((chunk ^ (row & 7)) << 4)) = o;
+                for (int k = 0; k < 4; ++k) {
+                    // channels 32 ch + 8 k + 2 cg, + 1: 16-byte chunk (4 (ch & 1) + k) of the 128-byte half row
+                    const int chunk = (ch & 1) * 4 + k;
+                    const uint32_t w_lo = pack_bf16(__uint_as_float(o[4 * k]) * inv_lo, __uint_as_float(o[4 * k + 1]) * inv_lo);
+                    const uint32_t w_hi = pack_bf16(__uint_as_float(o[4 * k + 2]) * inv_hi, __uint_as_float(o[4 * k + 3]) * inv_hi);
+                    *reinterpret_cast<uint32_t*>(so_lo + (ch >> 1) * QHALF_BYTES + ((chunk ^ sw_lo) << 4) + 4 * cg) = w_lo;
+                    *reinterpret_cast<uint32_t*>(so_hi + (ch >> 1) * QHALF_BYTES + ((chunk ^ sw_hi) << 4) + 4 * cg) = w_hi;
                 }
             }
             fence_proxy_async_smem();
         }
-        // the two warps of a query block meet, then one lane stores the block
+        // the four warps of a query block meet, then one lane stores the block
         const int qb_id = a;
-        named_barrier_sync(1 + qb_id, 64);
-        if (ok && (wl & 1) == 0 && lane == 0 && qblk(qb_id) * 64 < N) {
+        named_barrier_sync(1 + qb_id, 128);
+        if (ok && (wl & 1) == 0 && hf == 0 && lane == 0 && qblk(qb_id) * 64 < N) {
 #pragma unroll
             for (int dh = 0; dh < DH; ++dh)
                 tma_store_4d(&tmo, sQ + t * C::QTILE_BYTES + dh * QHALF_BYTES + (wl >> 1) * BLK_BYTES, dh * 64,
