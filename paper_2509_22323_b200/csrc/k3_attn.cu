@@ -166,29 +166,30 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     const uint32_t bPV = smem_u32(&ctl->pv_done[0]), bOD = smem_u32(&ctl->o_done[0]);        // [tile]: + 8 t
 
     // ---------------------------------------------------------------- setup
-    if (tid == 0) {
-        mbar_init(bQ, 1);
-        for (int s = 0; s < MAX_STAGES; ++s) {
-            mbar_init(bKF + 8 * s, 1);
-            mbar_init(bKE + 8 * s, 2);      // both tiles pass a stage before it is refilled
-            mbar_init(bVE + 8 * s, 2);
-        }
-        for (int s = 0; s < 4; ++s) {
-            mbar_init(bSF + 8 * s, 1);
-            mbar_init(bPF + 8 * s, 8);      // one arrival per softmax warp of the tile
-        }
-        for (int t = 0; t < 2; ++t) {
+    if (warp == 0) {                                    // one barrier group per lane
+        if (lane < MAX_STAGES) {
+            mbar_init(bKF + 8 * lane, 1);
+            mbar_init(bKE + 8 * lane, 2);   // both tiles pass a stage before it is refilled
+            mbar_init(bVE + 8 * lane, 2);
+        } else if (lane < MAX_STAGES + 4) {
+            mbar_init(bSF + 8 * (lane - MAX_STAGES), 1);
+            mbar_init(bPF + 8 * (lane - MAX_STAGES), 8);      // one arrival per softmax warp of the tile
+        } else if (lane < MAX_STAGES + 6) {
+            const int t = lane - MAX_STAGES - 4;
             mbar_init(bPV + 8 * t, 1);
             mbar_init(bOD + 8 * t, 1);
             mbar_init(smem_u32(&ctl->drain[t]), 1);
+        } else if (lane == MAX_STAGES + 6) {
+            mbar_init(bQ, 1);
+            ctl->abort_flag = 0;
+            ctl->n_u = 0;
+        } else if (lane == MAX_STAGES + 7) {
+            prefetch_tmap(&tmq);
+            prefetch_tmap(&tmk);
+            prefetch_tmap(&tmv);
+            prefetch_tmap(&tmo);
         }
-        ctl->abort_flag = 0;
-        ctl->n_u = 0;
         fence_mbar_init();
-        prefetch_tmap(&tmq);
-        prefetch_tmap(&tmk);
-        prefetch_tmap(&tmv);
-        prefetch_tmap(&tmo);
     }
     if (tid < 128) ctl->bm[tid / 32][tid % 32] = 0;
     if (warp == MMA_WARP0) {
@@ -198,6 +199,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     }
     __syncthreads();
 
+    // Key blocks known before the mask is read: a dense image keeps every block, and a mask of the selection kernel
+    // keeps the text blocks in every row, so the union list starts 0, 1, ... -- their K (and V) loads can start now.
+    const int n_early = (!INJECT && (slot < 0 || prm.bitmask32 != nullptr)) ? min(min(slot < 0 ? nb : g.n_text_blocks, nb), KS) : 0;
     // The Q tiles do not depend on the mask: start their loads before the union list is built.
     if (warp == PRODUCER_WARP && lane == 0) {
         mbar_arrive_expect_tx(bQ, 2 * C::QTILE_BYTES);
@@ -208,6 +212,18 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                 tma_load_4d(sQ + (ps2 ? (a & 1) : (a >> 1)) * C::QTILE_BYTES + dh * QHALF_BYTES +
                                 (ps2 ? (a >> 1) : (a & 1)) * BLK_BYTES, &tmq, bQ,
                             dh * 64, qblk(a) * 64, g.h0 + h, b);
+        // groups 0 .. n_early - 1 (group g = K(g) with V(g - 1)): first use of their stages, nothing to wait for
+        for (int gi = 0; gi < n_early; ++gi) {
+            mbar_arrive_expect_tx(bKF + 8 * gi, C::KV_BYTES + (gi > 0 ? C::KV_BYTES : 0));
+#pragma unroll
+            for (int dh = 0; dh < DH; ++dh)
+                tma_load_4d(sK + gi * C::KV_BYTES + dh * BLK_BYTES, &tmk, bKF + 8 * gi, dh * 64, gi * 64, g.h0 + h, b);
+            if (gi > 0) {
+#pragma unroll
+                for (int dh = 0; dh < DH; ++dh)
+                    tma_load_4d(sV + (gi - 1) * C::KV_BYTES + dh * BLK_BYTES, &tmv, bKF + 8 * gi, dh * 64, (gi - 1) * 64, g.h0 + h, b);
+            }
+        }
     }
 
     // ---------------------------------------------------------------- union of the four kept lists
@@ -287,7 +303,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             // issue S(g) = Q K(g)^T and O += P(g-1) V(g-1), so the pair completes ONE barrier (g_full[g % KS]) and
             // costs them one wait per key block instead of two.  Group 0 is K(0) alone, group n_u is V(n_u - 1)
             // alone.  A group is armed once both ring stages it fills have been released.
-            int g_issued = 0;
+            int g_issued = n_early;
             auto load_group = [&](int gi) -> bool {
                 const int s = gi % KS;
                 const bool has_k = gi < n_u, has_v = gi > 0;
@@ -313,7 +329,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                 return true;
             };
             bool ok = true;
-            for (int gi = 0; ok && n_u > 0 && gi <= n_u; ++gi) {
+            for (int gi = n_early; ok && n_u > 0 && gi <= n_u; ++gi) {
                 if (INJECT && gi == prm.stop_group) break;
                 ok = load_group(gi);
             }
