@@ -49,3 +49,18 @@ def test_single_process_aggregate_is_the_identity():
     import bench
     assert bench.aggregate(None, torch.device("cpu"), 1.5, 2.0, 3) == (1.5, 2.0, 3)
     assert bench.rank_step(0, 3) == 3 and bench.rank_step(2, 3) == 2003
+
+
+def test_bench_refuses_more_gpus_than_visible_and_mismatched_world_size():
+    """`python bench.py --gpus N` outside a launcher starts its N ranks itself; with fewer devices than that it
+    refuses (exit 2) before doing any work, and under a launcher --gpus must agree with WORLD_SIZE."""
+    import subprocess
+    n_dev = torch.cuda.device_count()
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", str(n_dev + 2), "--steps", "3"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 2 and "CUDA device" in r.stderr and r.stdout.strip() == ""
+    env["WORLD_SIZE"] = "4"
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "3"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode != 0 and "WORLD_SIZE=4" in r.stderr
