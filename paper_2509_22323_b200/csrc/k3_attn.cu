@@ -20,7 +20,8 @@
 //   warps 0-15  softmax, eight warps per tile and four per SM sub-partition: a warp owns 16 query rows, a
 //               thread a quarter of two rows (16x256b fragments; 32 scores per key block); fp32 online
 //               softmax with lazy rescale of O, P(n) written back over S(n) as bf16, final O / l store
-// TMEM: tile t owns columns [256 t, 256 t + 256): S(n) at 64 (n & 1), O at 128.
+// TMEM: tile t owns columns [256 t, 256 t + 256): S(n) at 64 (n mod NBUF), O behind the NBUF score buffers
+// (two of them and O at 128 for D = 128; three and O at 192 for D = 64, where the columns allow it).
 // Every mbarrier wait is bounded; a wait that runs out records RAPID3_ERR_TIMEOUT in the status
 // word and the CTA drains its copies, releases its TMEM and exits normally.
 #include "common.cuh"
@@ -28,6 +29,10 @@
 
 using namespace ptx;
 
+#ifndef RAPID3_NBUF64
+#define RAPID3_NBUF64 3
+#endif
+#define RAPID3_NBUF(D) ((D) == 64 ? (RAPID3_NBUF64) : 2)
 namespace {
 
 constexpr int SOFTMAX_WARPS = 16;
@@ -35,7 +40,6 @@ constexpr int PRODUCER_WARP = 16, MMA_WARP0 = 17;
 constexpr int NTHREADS = 32 * (SOFTMAX_WARPS + 3);
 constexpr int TMEM_COLS = 512;
 constexpr int TILE_COLS = 256;      // TMEM columns of one Q tile
-constexpr int O_COL = 128;
 constexpr int BLK_BYTES = 8192;     // 64 rows x 128 bytes: one 64-channel half of a 64-token block
 constexpr int QHALF_BYTES = 16384;  // one 64-channel half of a 128-row Q tile
 constexpr float RESCALE_LOG2 = 8.0f;
@@ -63,13 +67,15 @@ struct Cfg {
     static constexpr int KS = (D == 128) ? 4 : 8;           // K ring stages
     static constexpr int VS = (D == 128) ? 4 : 8;           // V ring stages
     static constexpr int DATA_BYTES = 2 * QTILE_BYTES + (KS + VS) * KV_BYTES;
+    static constexpr int NBUF = RAPID3_NBUF(D);             // score buffers (64 columns each) per tile
+    static constexpr int O_COL = 64 * NBUF;                 // O accumulator behind them: 64 NBUF + D <= 256 columns per tile
 };
 
 struct __align__(16) Ctl {
     unsigned long long q_full;
     unsigned long long k_full[MAX_STAGES], k_empty[MAX_STAGES];   // k_full[g % KS]: group g = K(g) and V(g - 1) have landed
     unsigned long long v_empty[MAX_STAGES];
-    unsigned long long s_full[2][2], p_full[2][2];
+    unsigned long long s_full[2][3], p_full[2][3];
     unsigned long long pv_done[2], o_done[2], drain[2];
     uint32_t tmem_base;
     int n_u;
@@ -97,7 +103,7 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
             const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo, const AttnParams prm) {
     using C = Cfg<D>;
-    constexpr int DH = C::DH, KS = C::KS, VS = C::VS;
+    constexpr int DH = C::DH, KS = C::KS, VS = C::VS, NBUF = C::NBUF, O_COL = C::O_COL;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
@@ -162,7 +168,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     const uint32_t bQ = smem_u32(&ctl->q_full);
     const uint32_t bKF = smem_u32(&ctl->k_full[0]), bKE = smem_u32(&ctl->k_empty[0]);
     const uint32_t bVE = smem_u32(&ctl->v_empty[0]);
-    const uint32_t bSF = smem_u32(&ctl->s_full[0][0]), bPF = smem_u32(&ctl->p_full[0][0]);   // [tile][buf]: + 16 t + 8 buf
+    const uint32_t bSF = smem_u32(&ctl->s_full[0][0]), bPF = smem_u32(&ctl->p_full[0][0]);   // [tile][buf]: + 24 t + 8 buf
     const uint32_t bPV = smem_u32(&ctl->pv_done[0]), bOD = smem_u32(&ctl->o_done[0]);        // [tile]: + 8 t
 
     // ---------------------------------------------------------------- setup
@@ -171,19 +177,19 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             mbar_init(bKF + 8 * lane, 1);
             mbar_init(bKE + 8 * lane, 2);   // both tiles pass a stage before it is refilled
             mbar_init(bVE + 8 * lane, 2);
-        } else if (lane < MAX_STAGES + 4) {
+        } else if (lane < MAX_STAGES + 6) {
             mbar_init(bSF + 8 * (lane - MAX_STAGES), 1);
             mbar_init(bPF + 8 * (lane - MAX_STAGES), 8);      // one arrival per softmax warp of the tile
-        } else if (lane < MAX_STAGES + 6) {
-            const int t = lane - MAX_STAGES - 4;
+        } else if (lane < MAX_STAGES + 8) {
+            const int t = lane - MAX_STAGES - 6;
             mbar_init(bPV + 8 * t, 1);
             mbar_init(bOD + 8 * t, 1);
             mbar_init(smem_u32(&ctl->drain[t]), 1);
-        } else if (lane == MAX_STAGES + 6) {
+        } else if (lane == MAX_STAGES + 8) {
             mbar_init(bQ, 1);
             ctl->abort_flag = 0;
             ctl->n_u = 0;
-        } else if (lane == MAX_STAGES + 7) {
+        } else if (lane == MAX_STAGES + 9) {
             prefetch_tmap(&tmq);
             prefetch_tmap(&tmk);
             prefetch_tmap(&tmv);
@@ -354,7 +360,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         const uint32_t tbase = tmem_base + t * TILE_COLS;
         const uint32_t tO = tbase + O_COL;
         const uint32_t qb = sQ + t * C::QTILE_BYTES;
-        const uint32_t bSFt = bSF + 16 * t, bPFt = bPF + 16 * t;
+        const uint32_t bSFt = bSF + 24 * t, bPFt = bPF + 24 * t;
         constexpr uint32_t idesc_qk = idesc_bf16(128, 64, 0, 0);
         constexpr uint32_t idesc_pv = idesc_bf16(128, D, 0, 1);
         int n_qk = 0, n_pv = 0;                        // blocks of this tile issued so far
@@ -366,7 +372,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             const bool use = ctl->u_flag[j] & tile_bits;
             if (use) {
                 tc_fence_after();
-                const uint32_t tS = tbase + 64 * (n_qk & 1);
+                const uint32_t tS = tbase + 64 * (n_qk % NBUF);
                 const uint32_t kb = sK + s * C::KV_BYTES;
                 if (leader) {
 #pragma unroll
@@ -374,7 +380,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                         mma_ss(tS, smem_desc_sw128(qb + (ks / 4) * QHALF_BYTES + (ks % 4) * 32, 16, 1024),
                                smem_desc_sw128(kb + (ks / 4) * BLK_BYTES + (ks % 4) * 32, 16, 1024), idesc_qk, ks > 0);
                     tc_commit(bKE + 8 * s);
-                    tc_commit(bSFt + 8 * (n_qk & 1));
+                    tc_commit(bSFt + 8 * (n_qk % NBUF));
                 }
                 ++n_qk;
             } else if (leader) {
@@ -384,17 +390,18 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             return true;
         };
         bool ok = (wait_warp(bQ, 0));
-        if (ok && n_u > 0) ok = k_step(0);
+        // the scores run NBUF - 1 key blocks ahead of the P V products
+        for (int j = 0; ok && j < NBUF - 1 && j <= n_u && n_u > 0; ++j) ok = k_step(j);
         for (int j = 0; ok && j < n_u; ++j) {
-            // S(n+1) reuses the buffer of P(n-1); the MMAs of the issuing thread execute in issue
-            // order, so it is written only after P(n-1) V has read it
-            if (!(ok = k_step(j + 1))) break;          // also brings V(j)
+            // S(n + NBUF - 1) reuses the buffer of P(n - 1); the MMAs of the issuing thread execute in issue
+            // order, so it is written only after P(n - 1) V has read it
+            if (j + NBUF - 1 <= n_u && !(ok = k_step(j + NBUF - 1))) break;          // group j + 1 brings V(j)
             const int s = j % VS;
             const bool use = ctl->u_flag[j] & tile_bits;
-            if (use && !(ok = (wait_warp(bPFt + 8 * (n_pv & 1), (n_pv >> 1) & 1)))) break;
+            if (use && !(ok = (wait_warp(bPFt + 8 * (n_pv % NBUF), (n_pv / NBUF) & 1)))) break;
             if (use) {
                 tc_fence_after();
-                const uint32_t tP = tbase + 64 * (n_pv & 1);
+                const uint32_t tP = tbase + 64 * (n_pv % NBUF);
                 const uint32_t vb = sV + s * C::KV_BYTES;
                 if (leader) {
 #pragma unroll
@@ -429,7 +436,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         const int row_lo = wl * 32 + hf * 16 + (lane >> 2);          // row of the 128-row tile; the second row is + 8
         const uint32_t lane_addr = tmem_base + ((uint32_t)(wl * 32 + hf * 16) << 16) + t * TILE_COLS;
         const uint32_t tO = lane_addr + O_COL;
-        const uint32_t bSFt = bSF + 16 * t, bPFt = bPF + 16 * t, bPVt = bPV + 8 * t;
+        const uint32_t bSFt = bSF + 24 * t, bPFt = bPF + 24 * t, bPVt = bPV + 8 * t;
         const float c2 = prm.scale_log2;
         const int tail_valid = N - (nb - 1) * 64;      // valid tokens of the last block (1..64)
         float m_lo = -INFINITY, m_hi = -INFINITY;      // reference maxima of the two rows
@@ -443,9 +450,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
             const int blk = ctl->u_blk[j];
             const bool act = (f >> a) & 1u;
             const int valid = (blk == nb - 1) ? tail_valid : 64;
-            const int buf = n & 1;
+            const int buf = n % NBUF;
             const uint32_t tS = lane_addr + 64 * buf;
-            if (!(ok = wait_warp(bSFt + 8 * buf, (n >> 1) & 1))) break;
+            if (!(ok = wait_warp(bSFt + 8 * buf, (n / NBUF) & 1))) break;
             tc_fence_after();
             uint32_t pk[16];
             if (act) {
