@@ -2,7 +2,7 @@
 //   pool_kernel   : one warp per (Q|K, image, head, 64-token block); 128-bit coalesced loads,
 //                   fp64 accumulation, mean over the valid tokens of the block.
 //                   HBM-bound: reads Q and K exactly once.
-//   scores_kernel : S[i][j] = Qbar[i,:] . Kbar[j,:] in fp64, rounded once to fp32.
+//   scores_kernel : S[i][j] = Qbar[i,:] . Kbar[j,:] in fp64 (fp64 mma.sync fragments), rounded once to fp32.
 #include "common.cuh"
 
 namespace {
@@ -71,69 +71,82 @@ __global__ void __launch_bounds__(128, 6) pool_kernel(const uint16_t* __restrict
     }
 }
 
-// T x T tile of S per CTA (T = 32 or 64), 16 x 16 threads, (T/16) x (T/16) outputs per thread, D in
-// chunks of 32 staged in shared memory; the next chunk is fetched into registers while the current
-// one is multiplied.  Every output accumulates its D products in ascending channel order.
+// D(8 x 8, fp64) += A(8 x 4, row) * B(4 x 8, col) on the fp64 tensor path (four times the rate of the fp64 FMA pipe
+// on this part).  Lane l holds a = A[l / 4][l % 4], b = B[l % 4][l / 4] and c0, c1 = D[l / 4][2 (l % 4) + {0, 1}].
+__device__ __forceinline__ void dmma_8x8x4(double& c0, double& c1, double a, double b) {
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                 : "+d"(c0), "+d"(c1)
+                 : "d"(a), "d"(b));
+}
+
+// T x T tile of S per CTA (T = 32; a multiple of 32), eight warps; a warp owns (T / 32) x (T / 16) fragments of 8 x 8 outputs.
+// D goes through shared memory in chunks of 32 channels (row stride 36 doubles: the fragment loads then touch every
+// bank pair twice, the minimum for 32 eight-byte lanes); the next chunk is fetched into registers while the
+// current one is multiplied.  Every output accumulates its products in ascending order of the four-channel groups.
 template <int T>
 __global__ void __launch_bounds__(256) scores_kernel(const double* __restrict__ pooled, TensorGeom g, int n_img,
                                                      float* __restrict__ scores, const DevPlan* __restrict__ plan) {
-    constexpr int R = T / 16;            // outputs per thread and dimension
+    constexpr int NI = T / 32;           // 8-row fragments per warp
+    constexpr int NJ = T / 16;           // 8-column fragments per warp
     constexpr int LD = T * 32 / 256;     // values a thread stages per operand and chunk
-    __shared__ double sq[T][33];
-    __shared__ double sk[T][33];
+    constexpr int LDS = 36;              // row stride of the staged chunks in doubles
+    __shared__ double sq[T][LDS];
+    __shared__ double sk[T][LDS];
     const int ph = blockIdx.z;                       // p * H + h
     if (plan && ph >= plan->sparse.n * g.H) return;
     const int i0 = blockIdx.y * T, j0 = blockIdx.x * T;
     const double* pq = pooled + (long long)ph * g.nb * g.D;
     const double* pk = pooled + ((long long)n_img * g.H + ph) * g.nb * g.D;
-    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
-    double acc[R][R];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32, gr = lane >> 2, c = lane & 3;
+    const int ri = (warp >> 1) * (8 * NI), cj = (warp & 1) * (8 * NJ);   // the warp's corner inside the tile
+    double acc[NI][NJ][2];
 #pragma unroll
-    for (int a = 0; a < R; ++a)
+    for (int a = 0; a < NI; ++a)
 #pragma unroll
-        for (int b = 0; b < R; ++b) acc[a][b] = 0.0;
+        for (int b = 0; b < NJ; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
     double rq[LD], rk[LD];
     auto fetch = [&](int d0) {
 #pragma unroll
         for (int u = 0; u < LD; ++u) {
-            const int e = threadIdx.x + u * 256, r = e / 32, c = e % 32;
-            rq[u] = (i0 + r < g.nb) ? pq[(long long)(i0 + r) * g.D + d0 + c] : 0.0;
-            rk[u] = (j0 + r < g.nb) ? pk[(long long)(j0 + r) * g.D + d0 + c] : 0.0;
+            const int e = threadIdx.x + u * 256, r = e / 32, cc = e % 32;
+            rq[u] = (i0 + r < g.nb) ? pq[(long long)(i0 + r) * g.D + d0 + cc] : 0.0;
+            rk[u] = (j0 + r < g.nb) ? pk[(long long)(j0 + r) * g.D + d0 + cc] : 0.0;
         }
     };
     fetch(0);
     for (int d0 = 0; d0 < g.D; d0 += 32) {
 #pragma unroll
         for (int u = 0; u < LD; ++u) {
-            const int e = threadIdx.x + u * 256, r = e / 32, c = e % 32;
-            sq[r][c] = rq[u];
-            sk[r][c] = rk[u];
+            const int e = threadIdx.x + u * 256, r = e / 32, cc = e % 32;
+            sq[r][cc] = rq[u];
+            sk[r][cc] = rk[u];
         }
         __syncthreads();
         if (d0 + 32 < g.D) fetch(d0 + 32);
-#pragma unroll 8
-        for (int d = 0; d < 32; ++d) {
-            double qv[R], kv[R];
 #pragma unroll
-            for (int a = 0; a < R; ++a) {
-                qv[a] = sq[ty + 16 * a][d];
-                kv[a] = sk[tx + 16 * a][d];
-            }
+        for (int d = 0; d < 32; d += 4) {
+            double qa[NI], kb[NJ];
 #pragma unroll
-            for (int a = 0; a < R; ++a)
+            for (int a = 0; a < NI; ++a) qa[a] = sq[ri + 8 * a + gr][d + c];
 #pragma unroll
-                for (int b = 0; b < R; ++b) acc[a][b] += qv[a] * kv[b];
+            for (int b = 0; b < NJ; ++b) kb[b] = sk[cj + 8 * b + gr][d + c];
+#pragma unroll
+            for (int a = 0; a < NI; ++a)
+#pragma unroll
+                for (int b = 0; b < NJ; ++b) dmma_8x8x4(acc[a][b][0], acc[a][b][1], qa[a], kb[b]);
         }
         __syncthreads();
     }
     float* so = scores + (long long)ph * g.nb * g.nb;
 #pragma unroll
-    for (int a = 0; a < R; ++a)
+    for (int a = 0; a < NI; ++a)
 #pragma unroll
-        for (int b = 0; b < R; ++b) {
-            const int i = i0 + ty + 16 * a, j = j0 + tx + 16 * b;
-            if (i < g.nb && j < g.nb) so[(long long)i * g.nb + j] = (float)acc[a][b];
-        }
+        for (int b = 0; b < NJ; ++b)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int i = i0 + ri + 8 * a + gr, j = j0 + cj + 8 * b + 2 * c + e;
+                if (i < g.nb && j < g.nb) so[(long long)i * g.nb + j] = (float)acc[a][b][e];
+            }
 }
 
 }  // namespace
@@ -151,15 +164,10 @@ cudaError_t launch_block_pool(const void* q, const void* k, const TensorGeom& g,
 
 cudaError_t launch_block_scores(const double* pooled, const TensorGeom& g, int n_img, float* scores,
                                 cudaStream_t s, const DevPlan* plan) {
-    // with a plan n_img is the capacity.  Long sequences take 64 x 64 tiles (half the shared-memory reads
-    // per product); short ones 32 x 32, which wastes less of the ragged edge and fills more SMs
-    if (g.nb >= 128) {
-        dim3 grid((g.nb + 63) / 64, (g.nb + 63) / 64, n_img * g.H);
-        scores_kernel<64><<<grid, 256, 0, s>>>(pooled, g, n_img, scores, plan);
-    } else {
-        dim3 grid((g.nb + 31) / 32, (g.nb + 31) / 32, n_img * g.H);
-        scores_kernel<32><<<grid, 256, 0, s>>>(pooled, g, n_img, scores, plan);
-    }
+    // with a plan n_img is the capacity.  32 x 32 tiles at every length: against 64 x 64 tiles they waste less of
+    // the ragged edge and fill the SMs more evenly (30 against 35 us at 264 blocks, where 64 x 64 pads 264 to 320)
+    dim3 grid((g.nb + 31) / 32, (g.nb + 31) / 32, n_img * g.H);
+    scores_kernel<32><<<grid, 256, 0, s>>>(pooled, g, n_img, scores, plan);
     return cudaGetLastError();
 }
 
