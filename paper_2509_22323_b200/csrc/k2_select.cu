@@ -1,9 +1,9 @@
 // K2: per (image, head, query-block row) forced + top-k block selection.
 // One warp per row.  The row of fp32 scores is staged in shared memory as order-preserving
 // 32-bit keys.  The k-th largest free candidate is found by a radix select over the key bits
-// (32 rounds of count-and-narrow, counts by lane-local sums and one warp reduction; rows with
-// fewer than ~100 candidates rank each candidate by counting the 64-bit (key, index) composites
-// that beat it instead); a free
+// (the bits all candidates share are skipped, the others go eight at a time through a 256-bin
+// histogram and a scan from the top; rows with at most 32 candidates rank each candidate by
+// counting the 64-bit (key, index) composites that beat it instead); a free
 // candidate is kept when its key is above that threshold, or equal to it and among the first
 // (lowest block index) of the equal ones still needed -- the order "score descending, index
 // ascending".  The bitmask is assembled with warp ballots and the ascending kept list with ballot
@@ -22,7 +22,7 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
                                                             int32_t* __restrict__ kept_idx,
                                                             int32_t* __restrict__ kept_cnt, int words32,
                                                             const DevPlan* __restrict__ plan, const HK hk) {
-    extern __shared__ unsigned long long srow[];          // [WARPS][nb_pad] 64-bit slots
+    extern __shared__ unsigned long long srow[];          // [WARPS][nb_pad] 64-bit slots, then [WARPS][256] histogram bins
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int nb = g.nb, ntb = g.n_text_blocks;
     const int nb_pad = (nb + 31) & ~31;
@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
     const bool text_row = i < ntb;
     const int n_free = max(nb - ntb - ((i >= ntb) ? 1 : 0), 0);
     const bool select = !text_row && k > 0 && k < n_free;
-    const bool radix = n_free > 96;                     // short rows: ranking by counting is cheaper than 32 rounds
+    const bool radix = n_free > 32;                     // short rows: ranking by counting is cheaper (measured: 63 candidates already favour the histogram)
     // key: unsigned integer with the same order as the float (-0 and +0 made equal), at least 2^23 for
     // any finite score.  Forced blocks and padding get key 0: they match no radix prefix (every trial
     // prefix has a bit set) and beat no candidate, so the loops below need no index tests.
@@ -60,18 +60,63 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
         else c64[j] = u ? (((unsigned long long)u << 32) | (uint32_t)(0xffffffffu - (uint32_t)j)) : 0ull;
     }
     __syncwarp();
-    // radix select of the k-th largest key among the free candidates
-    uint32_t prefix = 0u, mask = 0u;
+    // radix select of the k-th largest key among the free candidates: the bits all candidates share are skipped,
+    // the rest is taken eight bits at a time, each round a 256-bin histogram of the candidates that still match
+    // the prefix (shared-memory atomics) and a scan over the bins from the top
+    uint32_t prefix = 0u;
     int want = k;                                       // rank still looked for inside the prefix group
     if (select && radix) {
-        for (int bit = 31; bit >= 0; --bit) {
-            const uint32_t trial = prefix | (1u << bit), m2 = mask | (1u << bit);
-            int cnt = 0;
-            for (int j = lane; j < nb_pad; j += 32) cnt += ((s[j] & m2) == trial);
-            cnt = __reduce_add_sync(0xffffffffu, cnt);
-            if (cnt >= want) prefix = trial;
-            else want -= cnt;
-            mask = m2;
+        uint32_t* hist = reinterpret_cast<uint32_t*>(srow + WARPS * nb_pad) + warp * 256;
+        uint32_t k_and = 0xffffffffu, k_or = 0u;
+        for (int j = lane; j < nb_pad; j += 32) {
+            const uint32_t u = s[j];
+            if (u) { k_and &= u; k_or |= u; }
+        }
+        k_and = __reduce_and_sync(0xffffffffu, k_and);
+        k_or = __reduce_or_sync(0xffffffffu, k_or);
+        const uint32_t diff = k_and ^ k_or;             // bits in which two candidates differ
+        const int top = diff ? 32 - __clz(diff) : 0;    // only bits below `top` can differ
+        prefix = top >= 32 ? 0u : (k_or & ~((1u << top) - 1u));
+        for (int hi = top; hi > 0; hi -= 8) {           // digit = bits [lo, hi)
+            const int lo = max(hi - 8, 0);
+            const uint32_t dmask = (1u << (hi - lo)) - 1u;
+#pragma unroll
+            for (int b = 0; b < 8; ++b) hist[8 * lane + b] = 0u;
+            __syncwarp();
+            for (int j = lane; j < nb_pad; j += 32) {
+                const uint32_t u = s[j];
+                if (u && (hi >= 32 || (u >> hi) == (prefix >> hi))) atomicAdd(&hist[(u >> lo) & dmask], 1u);
+            }
+            __syncwarp();
+            // lane l owns bins 8 l .. 8 l + 7; S = candidates in its bins and all higher ones
+            uint32_t hloc[8], T = 0u;
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+                hloc[b] = hist[8 * lane + b];
+                T += hloc[b];
+            }
+            uint32_t S = T;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_down_sync(0xffffffffu, S, o);
+                if (lane + o < 32) S += v;
+            }
+            const int L = 31 - __clz(__ballot_sync(0xffffffffu, S >= (uint32_t)want));   // the lane whose bins hold the rank
+            int d_loc = -1;
+            uint32_t above_loc = 0u, running = S - T;
+#pragma unroll
+            for (int b = 7; b >= 0; --b) {
+                if (d_loc < 0 && running + hloc[b] >= (uint32_t)want) {
+                    d_loc = b;
+                    above_loc = running;
+                }
+                running += hloc[b];
+            }
+            const int d = __shfl_sync(0xffffffffu, 8 * lane + d_loc, L);
+            const uint32_t above = __shfl_sync(0xffffffffu, above_loc, L);
+            prefix |= (uint32_t)d << lo;
+            want -= (int)above;
+            __syncwarp();
         }
     }
     int32_t* out_idx = kept_idx + row * nb;
@@ -219,7 +264,7 @@ cudaError_t launch_select_mask_mass(const float* scores, const TensorGeom& g, co
     }
     const int words32 = 2 * ((g.nb + 63) / 64);
     const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
-    const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long);
+    const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long) + WARPS * 256 * sizeof(uint32_t);
     RowKeep rk;
     rk.k = row_keep;
     select_kernel<RowKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
@@ -233,7 +278,7 @@ cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const I
     const int nb_pad = (g.nb + 31) & ~31;
     const int words32 = 2 * ((g.nb + 63) / 64);
     const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
-    const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long);
+    const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long) + WARPS * 256 * sizeof(uint32_t);
     select_kernel<NoHeadKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
                                                         kept_cnt, words32, plan, NoHeadKeep());
     return cudaGetLastError();
@@ -245,7 +290,7 @@ cudaError_t launch_select_mask_heads(const float* scores, const TensorGeom& g, c
     const int nb_pad = (g.nb + 31) & ~31;
     const int words32 = 2 * ((g.nb + 63) / 64);
     const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
-    const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long);
+    const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long) + WARPS * 256 * sizeof(uint32_t);
     select_kernel<HeadKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
                                                        kept_cnt, words32, nullptr, hk);
     return cudaGetLastError();

@@ -3,7 +3,7 @@
 rapid3_select_mask is called on hand-made score tensors (no pooling in between, so the ties are
 exact on both sides) and compared with the oracle's selection bit for bit -- no near-tie
 allowance.  Both code paths of the kernel are covered: ranking by counting (rows with at most
-96 free candidates: nb = 5, 72) and the radix select (nb = 264, 1024)."""
+32 free candidates: nb = 5) and the radix select (nb = 72, 264, 1024)."""
 import os
 
 import numpy as np
