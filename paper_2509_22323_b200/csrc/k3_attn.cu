@@ -13,10 +13,10 @@
 //               the gathered K and V blocks into two rings of shared-memory stages; K(g) and
 //               V(g - 1), which the MMA warps need together, complete one barrier
 //   warps 17,18 UMMA issue, one warp per tile (warp 17 also owns the TMEM allocation).  S of a
-//               tile is double buffered in TMEM (2 x 64 fp32 columns): S(n+1) = Q K^T is issued
-//               before O += P(n) V, so the tensor pipe works on the next scores while the
+//               tile has NBUF buffers in TMEM (64 fp32 columns each): S(n + NBUF - 1) = Q K^T is
+//               issued before O += P(n) V, so the tensor pipe works on the next scores while the
 //               softmax warps are busy with the current ones.  Both warps walk the same union
-//               list one block ahead in K than in V; a stage is released when both have passed it
+//               list, K ahead of V; a stage is released when both have passed it
 //   warps 0-15  softmax, eight warps per tile and four per SM sub-partition: a warp owns 16 query rows, a
 //               thread a quarter of two rows (16x256b fragments; 32 scores per key block); fp32 online
 //               softmax with lazy rescale of O, P(n) written back over S(n) as bf16, final O / l store
@@ -29,10 +29,8 @@
 
 using namespace ptx;
 
-#ifndef RAPID3_NBUF64
-#define RAPID3_NBUF64 3
-#endif
-#define RAPID3_NBUF(D) ((D) == 64 ? (RAPID3_NBUF64) : 2)
+// score buffers per tile: three where the TMEM columns allow it (D = 64: 3 x 64 + 64 of O), else two
+#define RAPID3_NBUF(D) ((D) == 64 ? 3 : 2)
 namespace {
 
 constexpr int SOFTMAX_WARPS = 16;
