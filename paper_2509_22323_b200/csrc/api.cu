@@ -149,14 +149,15 @@ int get_map(rapid3_ctx* c, const void* base, CUtensorMap* out) {
 // `g` is the context's geometry or a copy of it narrowed to a range of heads.
 int attn_launch(rapid3_ctx* c, const TensorGeom& g, const void* q, const void* k, const void* v, void* out,
                 const ImgList& l, const int32_t* kept_idx, const int32_t* kept_cnt, const uint64_t* bitmask, float scale,
-                cudaStream_t st, const DevPlan* plan = nullptr, int n_cap = 0) {
+                cudaStream_t st, const DevPlan* plan = nullptr, int n_cap = 0, bool after_select = false) {
     CUtensorMap tq, tk, tv, to;
     int r;
     if ((r = get_map(c, q, &tq)) || (r = get_map(c, k, &tk)) || (r = get_map(c, v, &tv)) || (r = get_map(c, out, &to)))
         return r;
     {
         ProfScope ps(c, PROF_ATTN, st);
-        if (launch_attention(tq, tk, tv, to, g, l, kept_idx, kept_cnt, bitmask, scale, c->status, st, plan, n_cap) != cudaSuccess)
+        if (launch_attention(tq, tk, tv, to, g, l, kept_idx, kept_cnt, bitmask, scale, c->status, st, plan, n_cap, -1,
+                             after_select) != cudaSuccess)
             return RAPID3_ERR_CUDA;
     }
     c->launches += 1;
@@ -284,7 +285,7 @@ int rapid3_block_scores(rapid3_ctx* c, const void* q, const void* k, const int32
     }
     {
         ProfScope ps(c, PROF_SCORES, st);
-        if (launch_block_scores(c->pooled, c->g, n_img, scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+        if (launch_block_scores(c->pooled, c->g, n_img, scores, st, nullptr, true) != cudaSuccess) return RAPID3_ERR_CUDA;
     }
     c->launches += 2;
     return RAPID3_OK;
@@ -446,21 +447,21 @@ static int gated_step_impl(rapid3_ctx* c, const void* q, const void* k, const vo
         }
         {
             ProfScope ps(c, PROF_SCORES, st);
-            if (launch_block_scores(c->pooled, g, sparse.n, c->scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+            if (launch_block_scores(c->pooled, g, sparse.n, c->scores, st, nullptr, true) != cudaSuccess) return RAPID3_ERR_CUDA;
         }
         {
             ProfScope ps(c, PROF_SELECT, st);
             const cudaError_t e =
                 mass_scale ? launch_select_mask_mass(c->scores, g, sparse, share, *mass_scale, c->row_keep, c->bitmask,
                                                      c->kept_idx, c->kept_cnt, st)
-                : per_head ? launch_select_mask_heads(c->scores, g, sparse, hk, c->bitmask, c->kept_idx, c->kept_cnt, st)
-                           : launch_select_mask(c->scores, g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st);
+                : per_head ? launch_select_mask_heads(c->scores, g, sparse, hk, c->bitmask, c->kept_idx, c->kept_cnt, st, true)
+                           : launch_select_mask(c->scores, g, sparse, c->bitmask, c->kept_idx, c->kept_cnt, st, nullptr, 0, true);
             if (e != cudaSuccess) return RAPID3_ERR_CUDA;
         }
         c->launches += mass_scale ? 3 : 2;
     }
     return attn_launch(c, g, q, k, v, out, all, sparse.n ? c->kept_idx : nullptr, sparse.n ? c->kept_cnt : nullptr,
-                       sparse.n ? c->bitmask : nullptr, softmax_scale, st);
+                       sparse.n ? c->bitmask : nullptr, softmax_scale, st, nullptr, 0, sparse.n > 0 && !mass_scale);
 }
 
 int rapid3_gated_step(rapid3_ctx* c, const void* q, const void* k, const void* v, void* out,

@@ -58,20 +58,46 @@ struct TensorGeom {
     long long stride_b, stride_h, stride_n;   // elements
 };
 
+// Programmatic dependent launch: a kernel launched with `pdl` set may start while the kernel before it in the stream
+// is still running, and must call grid_dependency_wait() before it touches anything that kernel writes; the kernel
+// before it calls grid_dependency_launch() to let it start.  Both are no-ops in an ordinary launch.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl,
+                                 Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // K1: block means of Q and K (fp64) for the listed images, then S = Qbar . Kbar^T -> fp32.
 // With `plan` set the image list is read from device memory (plan->sparse) and the grid is sized
 // for `n_cap` images; CTAs beyond the planned count return at once.  pooled is [2][n_cap][H][nb][D].
 cudaError_t launch_block_pool(const void* q, const void* k, const TensorGeom& g, const ImgList& imgs,
                               double* pooled, cudaStream_t s, const DevPlan* plan = nullptr, int n_cap = 0);
+// `pdl`: the kernel before it in the stream is this library's pooling kernel (same for the launchers below: the
+// kernel named in their comment), so the launch may be a programmatic dependent one.
 cudaError_t launch_block_scores(const double* pooled, const TensorGeom& g, int n_img, float* scores,
-                                cudaStream_t s, const DevPlan* plan = nullptr);
+                                cudaStream_t s, const DevPlan* plan = nullptr, bool pdl = false);
 // K2: forced + top-k selection.
 cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const ImgList& imgs,
                                uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s,
-                               const DevPlan* plan = nullptr, int n_cap = 0);
+                               const DevPlan* plan = nullptr, int n_cap = 0, bool pdl = false);   // after the scores kernel
 cudaError_t launch_select_mask_heads(const float* scores, const TensorGeom& g, const ImgList& imgs,
                                      const HeadKeep& hk, uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt,
-                                     cudaStream_t s);
+                                     cudaStream_t s, bool pdl = false);                           // after the scores kernel
 // K2, cumulative-mass variant: row_keep[row] = smallest count of best free candidates holding a share
 // tau of the row's softmax mass (weights exp(scale * (S - row max)), fp64), then the top-k selection
 // at that count.
@@ -101,5 +127,6 @@ cudaError_t launch_plan(const int32_t* action_dev, const float* ratio_dev, int B
 cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, const CUtensorMap& tmv,
                              const CUtensorMap& tmo, const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
                              const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* status,
-                             cudaStream_t s, const DevPlan* plan = nullptr, int n_cap = 0, int inject_stop_group = -1);
+                             cudaStream_t s, const DevPlan* plan = nullptr, int n_cap = 0, int inject_stop_group = -1,
+                             int pdl = 0);   // 1: after the selection kernel, whose masks only the sparse images' thread blocks read
 cudaError_t attention_static_init();

@@ -25,6 +25,7 @@ __global__ void __launch_bounds__(128, 6) pool_kernel(const uint16_t* __restrict
     constexpr int ITERS = 64 / RPL;     // loads per lane
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int blk = blockIdx.x * 4 + warp, h = blockIdx.y;
+    grid_dependency_launch();                         // the scores kernel may be staged; it waits for this grid's end itself
     if (blk >= g.nb) return;
     const int which = blockIdx.z / n_cap;             // 0 = Q, 1 = K
     const int p = blockIdx.z - which * n_cap;
@@ -84,7 +85,7 @@ __device__ __forceinline__ void dmma_8x8x4(double& c0, double& c1, double a, dou
 // bank pair twice, the minimum for 32 eight-byte lanes); the next chunk is fetched into registers while the
 // current one is multiplied.  Every output accumulates its products in ascending order of the four-channel groups.
 template <int T>
-__global__ void __launch_bounds__(256) scores_kernel(const double* __restrict__ pooled, TensorGeom g, int n_img,
+__global__ void __launch_bounds__(256) scores_kernel(const double* pooled, TensorGeom g, int n_img,
                                                      float* __restrict__ scores, const DevPlan* __restrict__ plan) {
     constexpr int NI = T / 32;           // 8-row fragments per warp
     constexpr int NJ = T / 16;           // 8-column fragments per warp
@@ -93,6 +94,10 @@ __global__ void __launch_bounds__(256) scores_kernel(const double* __restrict__ 
     __shared__ double sq[T][LDS];
     __shared__ double sk[T][LDS];
     const int ph = blockIdx.z;                       // p * H + h
+    grid_dependency_launch();
+    // The block means come from the kernel before, which may still be running when this one starts: wait for its end,
+    // and read them past the L1 (ld.global.cg), whose lines no such wait is known to refresh.
+    grid_dependency_wait();
     if (plan && ph >= plan->sparse.n * g.H) return;
     const int i0 = blockIdx.y * T, j0 = blockIdx.x * T;
     const double* pq = pooled + (long long)ph * g.nb * g.D;
@@ -109,8 +114,8 @@ __global__ void __launch_bounds__(256) scores_kernel(const double* __restrict__ 
 #pragma unroll
         for (int u = 0; u < LD; ++u) {
             const int e = threadIdx.x + u * 256, r = e / 32, cc = e % 32;
-            rq[u] = (i0 + r < g.nb) ? pq[(long long)(i0 + r) * g.D + d0 + cc] : 0.0;
-            rk[u] = (j0 + r < g.nb) ? pk[(long long)(j0 + r) * g.D + d0 + cc] : 0.0;
+            rq[u] = (i0 + r < g.nb) ? __ldcg(pq + (long long)(i0 + r) * g.D + d0 + cc) : 0.0;
+            rk[u] = (j0 + r < g.nb) ? __ldcg(pk + (long long)(j0 + r) * g.D + d0 + cc) : 0.0;
         }
     };
     fetch(0);
@@ -163,12 +168,11 @@ cudaError_t launch_block_pool(const void* q, const void* k, const TensorGeom& g,
 }
 
 cudaError_t launch_block_scores(const double* pooled, const TensorGeom& g, int n_img, float* scores,
-                                cudaStream_t s, const DevPlan* plan) {
+                                cudaStream_t s, const DevPlan* plan, bool pdl) {
     // with a plan n_img is the capacity.  32 x 32 tiles at every length: against 64 x 64 tiles they waste less of
     // the ragged edge and fill the SMs more evenly (30 against 35 us at 264 blocks, where 64 x 64 pads 264 to 320)
     dim3 grid((g.nb + 31) / 32, (g.nb + 31) / 32, n_img * g.H);
-    scores_kernel<32><<<grid, 256, 0, s>>>(pooled, g, n_img, scores, plan);
-    return cudaGetLastError();
+    return launch_kernel(scores_kernel<32>, grid, dim3(256), 0, s, pdl, pooled, g, n_img, scores, plan);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -257,7 +261,7 @@ extern "C" int rapid3_block_scores_static(const rapid3_shape* s, const void* q, 
     // every element of the used part of the scratch is written by the pooling kernel before the
     // scoring kernel reads it, so nothing has to be cleared between calls
     if (launch_block_pool(q, k, g, l, scratch, st) != cudaSuccess) return RAPID3_ERR_CUDA;
-    if (launch_block_scores(scratch, g, n_img, scores, st) != cudaSuccess) return RAPID3_ERR_CUDA;
+    if (launch_block_scores(scratch, g, n_img, scores, st, nullptr, true) != cudaSuccess) return RAPID3_ERR_CUDA;
     return RAPID3_OK;
 }
 

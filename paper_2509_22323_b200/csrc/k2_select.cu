@@ -17,7 +17,7 @@ constexpr int WARPS = 4;
 // HK = NoHeadKeep: one keep count per image.  HK = HeadKeep: one per (image, head), passed by value.
 // HK = RowKeep: one per row, read from device memory.
 template <typename HK>
-__global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restrict__ scores, TensorGeom g,
+__global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* scores, TensorGeom g,
                                                             ImgList imgs, uint32_t* __restrict__ bitmask32,
                                                             int32_t* __restrict__ kept_idx,
                                                             int32_t* __restrict__ kept_cnt, int words32,
@@ -27,6 +27,8 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
     const int nb = g.nb, ntb = g.n_text_blocks;
     const int nb_pad = (nb + 31) & ~31;
     const long long row = (long long)blockIdx.x * WARPS + warp;        // (p * H + h) * nb + i
+    grid_dependency_launch();
+    grid_dependency_wait();                             // the scores come from the kernel before, which may still be running
     const long long n_rows = (long long)(plan ? plan->sparse.n : imgs.n) * g.H * nb;
     if (row >= n_rows) return;
     const int i = (int)(row % nb);
@@ -51,7 +53,7 @@ __global__ void __launch_bounds__(WARPS * 32) select_kernel(const float* __restr
     for (int j = lane; j < nb_pad; j += 32) {
         uint32_t u = 0u;
         if (j < nb && j >= ntb && j != i) {
-            u = __float_as_uint(src[j]);
+            u = __float_as_uint(__ldcg(src + j));              // past the L1: see the wait above
             if (u == 0x80000000u) u = 0u;
             u ^= (u >> 31) ? 0xffffffffu : 0x80000000u;
         }
@@ -273,27 +275,26 @@ cudaError_t launch_select_mask_mass(const float* scores, const TensorGeom& g, co
 }
 
 cudaError_t launch_select_mask(const float* scores, const TensorGeom& g, const ImgList& imgs, uint64_t* bitmask,
-                               int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s, const DevPlan* plan, int n_cap) {
+                               int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s, const DevPlan* plan, int n_cap,
+                               bool pdl) {
     const long long n_rows = (long long)(plan ? n_cap : imgs.n) * g.H * g.nb;
     const int nb_pad = (g.nb + 31) & ~31;
     const int words32 = 2 * ((g.nb + 63) / 64);
     const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
     const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long) + WARPS * 256 * sizeof(uint32_t);
-    select_kernel<NoHeadKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
-                                                        kept_cnt, words32, plan, NoHeadKeep());
-    return cudaGetLastError();
+    return launch_kernel(select_kernel<NoHeadKeep>, dim3(grid), dim3(WARPS * 32), smem, s, pdl, scores, g, imgs,
+                         reinterpret_cast<uint32_t*>(bitmask), kept_idx, kept_cnt, words32, plan, NoHeadKeep());
 }
 
 cudaError_t launch_select_mask_heads(const float* scores, const TensorGeom& g, const ImgList& imgs, const HeadKeep& hk,
-                                     uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s) {
+                                     uint64_t* bitmask, int32_t* kept_idx, int32_t* kept_cnt, cudaStream_t s, bool pdl) {
     const long long n_rows = (long long)imgs.n * g.H * g.nb;
     const int nb_pad = (g.nb + 31) & ~31;
     const int words32 = 2 * ((g.nb + 63) / 64);
     const unsigned grid = (unsigned)((n_rows + WARPS - 1) / WARPS);
     const size_t smem = (size_t)WARPS * nb_pad * sizeof(unsigned long long) + WARPS * 256 * sizeof(uint32_t);
-    select_kernel<HeadKeep><<<grid, WARPS * 32, smem, s>>>(scores, g, imgs, reinterpret_cast<uint32_t*>(bitmask), kept_idx,
-                                                       kept_cnt, words32, nullptr, hk);
-    return cudaGetLastError();
+    return launch_kernel(select_kernel<HeadKeep>, dim3(grid), dim3(WARPS * 32), smem, s, pdl, scores, g, imgs,
+                         reinterpret_cast<uint32_t*>(bitmask), kept_idx, kept_cnt, words32, static_cast<const DevPlan*>(nullptr), hk);
 }
 
 

@@ -74,7 +74,7 @@ struct __align__(16) Ctl {
     unsigned long long k_full[MAX_STAGES], k_empty[MAX_STAGES];   // k_full[g % KS]: group g = K(g) and V(g - 1) have landed
     unsigned long long v_empty[MAX_STAGES];
     unsigned long long s_full[2][3], p_full[2][3];
-    unsigned long long pv_done[2], o_done[2], drain[2];
+    unsigned long long pv_done[2][3], o_done[2], drain[2];
     uint32_t tmem_base;
     int n_u;
     volatile int abort_flag;
@@ -167,7 +167,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     const uint32_t bKF = smem_u32(&ctl->k_full[0]), bKE = smem_u32(&ctl->k_empty[0]);
     const uint32_t bVE = smem_u32(&ctl->v_empty[0]);
     const uint32_t bSF = smem_u32(&ctl->s_full[0][0]), bPF = smem_u32(&ctl->p_full[0][0]);   // [tile][buf]: + 24 t + 8 buf
-    const uint32_t bPV = smem_u32(&ctl->pv_done[0]), bOD = smem_u32(&ctl->o_done[0]);        // [tile]: + 8 t
+    const uint32_t bPV = smem_u32(&ctl->pv_done[0][0]);                                      // [tile][buf] as well
+    const uint32_t bOD = smem_u32(&ctl->o_done[0]);                                          // [tile]: + 8 t
 
     // ---------------------------------------------------------------- setup
     if (warp == 0) {                                    // one barrier group per lane
@@ -178,9 +179,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         } else if (lane < MAX_STAGES + 6) {
             mbar_init(bSF + 8 * (lane - MAX_STAGES), 1);
             mbar_init(bPF + 8 * (lane - MAX_STAGES), 8);      // one arrival per softmax warp of the tile
+            mbar_init(bPV + 8 * (lane - MAX_STAGES), 1);
         } else if (lane < MAX_STAGES + 8) {
             const int t = lane - MAX_STAGES - 6;
-            mbar_init(bPV + 8 * t, 1);
             mbar_init(bOD + 8 * t, 1);
             mbar_init(smem_u32(&ctl->drain[t]), 1);
         } else if (lane == MAX_STAGES + 8) {
@@ -234,19 +235,24 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     // bm[a] = bit set of the key blocks query block a keeps: copied from the bitmask when the
     // caller has one, else rebuilt from the kept list; every block is kept for a dense image.
     const int nw = (nb + 31) >> 5;
+    // Launched as a dependent of the selection kernel, a thread block of a sparse image waits here for the masks; one of
+    // a dense image reads nothing of them and runs on (its wait comes at the end, so that the grid as a whole still
+    // ends after the selection kernel).  The masks are read past the L1 (ld.global.cg): this thread block may have
+    // started before they were written, and an L1 line of an earlier step must not answer.
+    if (slot >= 0) grid_dependency_wait();
     if (slot >= 0 && prm.bitmask32 != nullptr) {
         if (tid < 4 * nw) {
             const int a = tid / nw, w = tid - a * nw;
             if (qblk(a) < nb)
-                ctl->bm[a][w] = prm.bitmask32[(((long long)slot * g.H + h) * nb + qblk(a)) * prm.words32 + w];
+                ctl->bm[a][w] = __ldcg(prm.bitmask32 + (((long long)slot * g.H + h) * nb + qblk(a)) * prm.words32 + w);
         }
     } else if (slot >= 0 && prm.kept_idx != nullptr) {
         for (int a = 0; a < 4 && qblk(a) < nb; ++a) {
             const long long row = ((long long)slot * g.H + h) * nb + qblk(a);
-            const int cnt = min(max(prm.kept_cnt[row], 0), nb);
+            const int cnt = min(max(__ldcg(prm.kept_cnt + row), 0), nb);
             const int32_t* lst = prm.kept_idx + row * nb;
             for (int e = tid; e < cnt; e += NTHREADS) {
-                const int j = lst[e];
+                const int j = __ldcg(lst + e);
                 if ((unsigned)j < (unsigned)nb) atomicOr(&ctl->bm[a][j >> 5], 1u << (j & 31));
                 else atomicExch(prm.status, RAPID3_ERR_BAD_LIST);
             }
@@ -407,9 +413,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                         mma_ts(tO, tP + ks * 8, smem_desc_sw128(vb + ks * 2048, BLK_BYTES, 1024), idesc_pv,
                                (n_pv > 0 || ks > 0) ? 1u : 0u);
                     tc_commit(bVE + 8 * s);
-                    // pv_done advances one phase per block of the tile (the rescale path waits on the
-                    // previous block's phase); the epilogue may lag, so it has its own barrier
-                    tc_commit(bPV + 8 * t);
+                    // pv_done has one barrier per score buffer, like s_full and p_full: the softmax warps run up
+                    // to NBUF - 1 blocks ahead of these products, and the parity of a single barrier cannot tell
+                    // "block n - 1 is done" from "block n - 3 is done".  The rescale path waits on the previous
+                    // block's buffer; the epilogue may lag, so it has its own barrier.
+                    tc_commit(bPV + 24 * t + 8 * (n_pv % NBUF));
                 }
                 ++n_pv;
             } else if (leader) {
@@ -434,7 +442,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         const int row_lo = wl * 32 + hf * 16 + (lane >> 2);          // row of the 128-row tile; the second row is + 8
         const uint32_t lane_addr = tmem_base + ((uint32_t)(wl * 32 + hf * 16) << 16) + t * TILE_COLS;
         const uint32_t tO = lane_addr + O_COL;
-        const uint32_t bSFt = bSF + 24 * t, bPFt = bPF + 24 * t, bPVt = bPV + 8 * t;
+        const uint32_t bSFt = bSF + 24 * t, bPFt = bPF + 24 * t, bPVt = bPV + 24 * t;
         const float c2 = prm.scale_log2;
         const int tail_valid = N - (nb - 1) * 64;      // valid tokens of the last block (1..64)
         float m_lo = -INFINITY, m_hi = -INFINITY;      // reference maxima of the two rows
@@ -501,8 +509,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                         const bool g_lo = (mx_lo - m_lo) * c2 > RESCALE_LOG2, g_hi = (mx_hi - m_hi) * c2 > RESCALE_LOG2;   // true from -inf
                         const bool f_lo = g_lo && m_lo != -INFINITY, f_hi = g_hi && m_hi != -INFINITY;   // O holds something to rescale
                         if (__any_sync(0xffffffffu, f_lo || f_hi)) {
-                            // O must be at rest: wait for P(n-1) V
-                            if (!(ok = wait_warp(bPVt, (n - 1) & 1))) break;
+                            // O must be at rest: wait for P(n-1) V, which by the issue order of the products also
+                            // tells that every earlier one is done
+                            if (!(ok = wait_warp(bPVt + 8 * ((n - 1) % NBUF), ((n - 1) / NBUF) & 1))) break;
                             tc_fence_after();
                             const float a_lo = f_lo ? ex2((m_lo - mx_lo) * c2) : 1.f, a_hi = f_hi ? ex2((m_hi - mx_hi) * c2) : 1.f;
                             l0 *= a_lo; l1 *= a_lo; l2 *= a_hi; l3 *= a_hi;
@@ -585,6 +594,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     }
 
     // ---------------------------------------------------------------- teardown
+    if (slot < 0) grid_dependency_wait();
     tc_fence_before();
     __syncthreads();
     if (warp >= MMA_WARP0) {
@@ -629,7 +639,7 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
                              const CUtensorMap& tmo,
                              const TensorGeom& g, const ImgList& imgs, const int32_t* kept_idx,
                              const int32_t* kept_cnt, const uint64_t* bitmask, float softmax_scale, int* status,
-                             cudaStream_t s, const DevPlan* plan, int n_cap, int inject_stop_group) {
+                             cudaStream_t s, const DevPlan* plan, int n_cap, int inject_stop_group, int pdl) {
     if (!g_attr_set) {
         cudaError_t e = attention_static_init();
         if (e != cudaSuccess) return e;
@@ -655,9 +665,9 @@ cudaError_t launch_attention(const CUtensorMap& tmq, const CUtensorMap& tmk, con
         else
             attn_kernel<64, true><<<grid, NTHREADS, attn_smem_bytes<64>(), s>>>(tmq, tmk, tmv, tmo, prm);
     } else if (g.D == 128) {
-        attn_kernel<128><<<grid, NTHREADS, attn_smem_bytes<128>(), s>>>(tmq, tmk, tmv, tmo, prm);
+        return launch_kernel(attn_kernel<128>, grid, dim3(NTHREADS), attn_smem_bytes<128>(), s, pdl != 0, tmq, tmk, tmv, tmo, prm);
     } else {
-        attn_kernel<64><<<grid, NTHREADS, attn_smem_bytes<64>(), s>>>(tmq, tmk, tmv, tmo, prm);
+        return launch_kernel(attn_kernel<64>, grid, dim3(NTHREADS), attn_smem_bytes<64>(), s, pdl != 0, tmq, tmk, tmv, tmo, prm);
     }
     return cudaGetLastError();
 }
