@@ -74,7 +74,7 @@ struct __align__(16) Ctl {
     unsigned long long k_full[MAX_STAGES], k_empty[MAX_STAGES];   // k_full[g % KS]: group g = K(g) and V(g - 1) have landed
     unsigned long long v_empty[MAX_STAGES];
     unsigned long long s_full[2][3], p_full[2][3];
-    unsigned long long pv_done[2][3], o_done[2], drain[2];
+    unsigned long long pv_done[2][2], o_done[2], drain[2];
     uint32_t tmem_base;
     int n_u;
     volatile int abort_flag;
@@ -167,7 +167,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     const uint32_t bKF = smem_u32(&ctl->k_full[0]), bKE = smem_u32(&ctl->k_empty[0]);
     const uint32_t bVE = smem_u32(&ctl->v_empty[0]);
     const uint32_t bSF = smem_u32(&ctl->s_full[0][0]), bPF = smem_u32(&ctl->p_full[0][0]);   // [tile][buf]: + 24 t + 8 buf
-    const uint32_t bPV = smem_u32(&ctl->pv_done[0][0]);                                      // [tile][buf] as well
+    const uint32_t bPV = smem_u32(&ctl->pv_done[0][0]);                                      // [tile][block parity]: + 16 t + 8 (n & 1)
     const uint32_t bOD = smem_u32(&ctl->o_done[0]);                                          // [tile]: + 8 t
 
     // ---------------------------------------------------------------- setup
@@ -179,9 +179,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         } else if (lane < MAX_STAGES + 6) {
             mbar_init(bSF + 8 * (lane - MAX_STAGES), 1);
             mbar_init(bPF + 8 * (lane - MAX_STAGES), 8);      // one arrival per softmax warp of the tile
-            mbar_init(bPV + 8 * (lane - MAX_STAGES), 1);
         } else if (lane < MAX_STAGES + 8) {
             const int t = lane - MAX_STAGES - 6;
+            mbar_init(bPV + 16 * t, 1);
+            mbar_init(bPV + 16 * t + 8, 1);
             mbar_init(bOD + 8 * t, 1);
             mbar_init(smem_u32(&ctl->drain[t]), 1);
         } else if (lane == MAX_STAGES + 8) {
@@ -236,8 +237,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     // caller has one, else rebuilt from the kept list; every block is kept for a dense image.
     const int nw = (nb + 31) >> 5;
     // Launched as a dependent of the selection kernel, a thread block of a sparse image waits here for the masks; one of
-    // a dense image reads nothing of them and runs on (its wait comes at the end, so that the grid as a whole still
-    // ends after the selection kernel).  The masks are read past the L1 (ld.global.cg): this thread block may have
+    // a dense image reads nothing of them and runs on (an idle lane of its producer warp waits instead, so that the
+    // grid as a whole still ends after the selection kernel).  The masks are read past the L1 (ld.global.cg): this thread block may have
     // started before they were written, and an L1 line of an earlier step must not answer.
     if (slot >= 0) grid_dependency_wait();
     if (slot >= 0 && prm.bitmask32 != nullptr) {
@@ -308,6 +309,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
 
     if (warp == PRODUCER_WARP) {
         // ------------------------------------------------------------ producer
+        if (slot < 0 && lane == 1) grid_dependency_wait();   // see above; off every critical path
         if (lane == 0) {
             // Group g = K block g together with V block g - 1: the MMA warps need exactly that pair before they
             // issue S(g) = Q K(g)^T and O += P(g-1) V(g-1), so the pair completes ONE barrier (g_full[g % KS]) and
@@ -413,11 +415,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                         mma_ts(tO, tP + ks * 8, smem_desc_sw128(vb + ks * 2048, BLK_BYTES, 1024), idesc_pv,
                                (n_pv > 0 || ks > 0) ? 1u : 0u);
                     tc_commit(bVE + 8 * s);
-                    // pv_done has one barrier per score buffer, like s_full and p_full: the softmax warps run up
-                    // to NBUF - 1 blocks ahead of these products, and the parity of a single barrier cannot tell
-                    // "block n - 1 is done" from "block n - 3 is done".  The rescale path waits on the previous
-                    // block's buffer; the epilogue may lag, so it has its own barrier.
-                    tc_commit(bPV + 24 * t + 8 * (n_pv % NBUF));
+                    // pv_done: two barriers per tile, for the even and the odd blocks.  The softmax warps run up
+                    // to NBUF - 1 <= 2 blocks ahead of these products, and the parity of one barrier taking every
+                    // block could not tell "block n - 1 is done" from "block n - 3 is done"; with two, the one the
+                    // rescale path waits on (block n - 1's) can only be one phase behind, because S(n) exists only
+                    // once the product of block n - NBUF is over.  The epilogue may lag, so it has its own barrier.
+                    tc_commit(bPV + 16 * t + 8 * (n_pv & 1));
                 }
                 ++n_pv;
             } else if (leader) {
@@ -442,7 +445,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         const int row_lo = wl * 32 + hf * 16 + (lane >> 2);          // row of the 128-row tile; the second row is + 8
         const uint32_t lane_addr = tmem_base + ((uint32_t)(wl * 32 + hf * 16) << 16) + t * TILE_COLS;
         const uint32_t tO = lane_addr + O_COL;
-        const uint32_t bSFt = bSF + 24 * t, bPFt = bPF + 24 * t, bPVt = bPV + 24 * t;
+        const uint32_t bSFt = bSF + 24 * t, bPFt = bPF + 24 * t, bPVt = bPV + 16 * t;
         const float c2 = prm.scale_log2;
         const int tail_valid = N - (nb - 1) * 64;      // valid tokens of the last block (1..64)
         float m_lo = -INFINITY, m_hi = -INFINITY;      // reference maxima of the two rows
@@ -511,7 +514,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                         if (__any_sync(0xffffffffu, f_lo || f_hi)) {
                             // O must be at rest: wait for P(n-1) V, which by the issue order of the products also
                             // tells that every earlier one is done
-                            if (!(ok = wait_warp(bPVt + 8 * ((n - 1) % NBUF), ((n - 1) / NBUF) & 1))) break;
+                            if (!(ok = wait_warp(bPVt + 8 * ((n - 1) & 1), ((n - 1) >> 1) & 1))) break;
                             tc_fence_after();
                             const float a_lo = f_lo ? ex2((m_lo - mx_lo) * c2) : 1.f, a_hi = f_hi ? ex2((m_hi - mx_hi) * c2) : 1.f;
                             l0 *= a_lo; l1 *= a_lo; l2 *= a_hi; l3 *= a_hi;
@@ -594,7 +597,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
     }
 
     // ---------------------------------------------------------------- teardown
-    if (slot < 0) grid_dependency_wait();
     tc_fence_before();
     __syncthreads();
     if (warp >= MMA_WARP0) {
