@@ -70,3 +70,54 @@ def test_queued_scoring_calls_equal_calls_run_alone():
     torch.cuda.synchronize()
     for s in range(3):
         assert torch.equal(got[s], alone[s]), f"scoring call {s}"
+
+
+def _variants(wl, n_sets):
+    """name -> function (ctx, set index, q, k, v, out) issuing one step of that entry point."""
+    acts, ratios = inputs.make_actions(wl, 0)
+    g = torch.Generator(device="cpu").manual_seed(4242)
+    head_ratios = [[float(min(1.0, max(0.05, r * f))) for f in (0.5 + torch.rand(wl.heads, generator=g)).tolist()]
+                   for r in ratios]
+    shares = [0.5 + 0.4 * i / max(1, wl.batch - 1) for i in range(wl.batch)]
+    acts_dev = torch.tensor(acts, dtype=torch.int32, device=DEV)
+    ratios_dev = torch.tensor(ratios, dtype=torch.float32, device=DEV)
+    q_gain = (0.5 + torch.rand(wl.head_dim, generator=g)).to(DEV)
+    k_gain = (0.5 + torch.rand(wl.head_dim, generator=g)).to(DEV)
+    produced = [(torch.empty((wl.batch, wl.heads, wl.n_tokens, wl.head_dim), dtype=torch.bfloat16, device=DEV),
+                 torch.empty((wl.batch, wl.heads, wl.n_tokens, wl.head_dim), dtype=torch.bfloat16, device=DEV))
+                for _ in range(n_sets)]
+    return {
+        "heads": lambda c, s, q, k, v, o: c.rapid3_gated_step_heads(q, k, v, o, acts, head_ratios, wl.softmax_scale),
+        "mass": lambda c, s, q, k, v, o: c.rapid3_gated_step_mass(q, k, v, o, acts, shares, wl.softmax_scale,
+                                                                  wl.softmax_scale),
+        "device": lambda c, s, q, k, v, o: c.rapid3_gated_step_device(q, k, v, o, acts_dev, ratios_dev,
+                                                                      wl.softmax_scale),
+        "fused": lambda c, s, q, k, v, o: c.rapid3_gated_step_fused(q, k, v, q_gain, k_gain, None, 1e-6,
+                                                                    produced[s][0], produced[s][1], o, acts, ratios,
+                                                                    wl.softmax_scale),
+    }
+
+
+@pytest.mark.parametrize("variant", ["heads", "mass", "device", "fused"])
+@pytest.mark.parametrize("name", ["sd3_1024", "flux_1024"])
+def test_queued_steps_of_the_other_entry_points(name, variant):
+    wl = inputs.WORKLOADS[name]
+    n_sets = 3
+    sets = [inputs.make_qkv(wl, s, device=DEV) for s in range(n_sets)]
+    step = _variants(wl, n_sets)[variant]
+    alone = []
+    for s in range(n_sets):
+        ctx = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
+        out = torch.zeros_like(sets[0][0])
+        step(ctx, s, *sets[s], out)
+        torch.cuda.synchronize()
+        assert ctx.last_status() == 0
+        alone.append(out)
+    ctx = binding.Context(wl.batch, wl.heads, wl.head_dim, wl.n_text, wl.n_image)
+    outs = [torch.zeros_like(sets[0][0]) for _ in range(n_sets)]
+    for i in range(4 * n_sets):
+        step(ctx, i % n_sets, *sets[i % n_sets], outs[i % n_sets])
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    for s in range(n_sets):
+        assert torch.equal(outs[s].view(torch.int16), alone[s].view(torch.int16)), f"{name} {variant}: input set {s}"
