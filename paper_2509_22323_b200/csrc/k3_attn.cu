@@ -463,6 +463,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
         bool ok = true;
         uint32_t r[32];
         int n = 0;                                     // blocks of this tile so far
+        bool seeded = false;                           // the rows' reference maxima have been set (warp-uniform: a warp's rows share a query block)
         for (int j = 0; j < n_u; ++j) {
             const uint32_t f = ctl->u_flag[j];
             if (!(f & tile_bits)) continue;            // neither query block of the tile kept it
@@ -490,10 +491,25 @@ attn_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUt
                 // One pass over the 32 scores gives P = 2^(S c2 - m c2) (packed to bf16), the block's partial
                 // row sums and the thread's share of the block's row maxima.  The pass runs with the reference
                 // maxima as they stand, so the exponentials do not wait for this block's maximum; only when a
-                // row's maximum has grown by more than 2^8 (rare after the first blocks, always at the first
-                // block) O and l are rescaled and the pass is repeated.
+                // row's maximum has grown by more than 2^8 (rare after the first blocks) O and l are rescaled
+                // and the pass is repeated.
                 float b0, b1, b2, b3;
                 bool redo;
+                if (!seeded) {
+                    // the first block this query block keeps: take the rows' maxima before the pass instead of running
+                    // the pass twice (from -inf every row "grows")
+                    float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        mx_lo = max3(mx_lo, __uint_as_float(r[4 * k]), __uint_as_float(r[4 * k + 1]));
+                        mx_hi = max3(mx_hi, __uint_as_float(r[4 * k + 2]), __uint_as_float(r[4 * k + 3]));
+                    }
+                    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+                    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+                    m_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+                    m_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+                    seeded = true;
+                }
                 do {
                     const float ms_lo = m_lo * c2, ms_hi = m_hi * c2;
                     float mx_lo = -INFINITY, mx_hi = -INFINITY;
