@@ -34,7 +34,7 @@ METRIC = "block-sparse joint-attn ms/call & effective TFLOPS (kept tiles) vs bf1
 UNIT = "TFLOP/s (kept tiles)"
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu summary in
 # profiles/ (null until a capture of that workload exists)
-ATTN_DRAM_BYTES_PER_LAUNCH = {"flux_1024": 417898496, "flux_2048": 577933824, "sd3_1024": 93194752}
+ATTN_DRAM_BYTES_PER_LAUNCH = {"flux_1024": 423511808, "flux_2048": 579094784, "sd3_1024": 94116608}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
